@@ -1,0 +1,206 @@
+"""CPU oracle for one S3GD-MV compression / aggregation / update step.
+
+TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct
+statement of what the hot path computes.  It shares no code with the CUDA
+library and must never be imported by it; only the tests, the smoke check and
+the benchmark's CPU-baseline leg may call it.
+
+What is computed (paper: Park & Lee, "Sparse-SignSGD with Majority Vote"):
+
+* TopK / TopKSign (Section 2.1, Eq. (3) ``TopK`` and Eq. (4) ``TopKSign``):
+  keep the K entries of largest magnitude, replace them by their sign.
+* Majority vote (Section 2.2, "Majority vote" paragraph and Algorithm 1):
+  sgn of the sum over workers of the ternary vectors; coordinates nobody voted
+  on, and exact ties, stay 0 because sgn(0) = 0 in the paper's definition.
+* Model update (Section 2.2, Eq. (7)): x <- x - delta * vote.
+
+Readings where the paper is silent (all listed in the design notes):
+
+* magnitude order is the unsigned order of the fp32 bit pattern with the sign
+  bit cleared (so denormals, Inf and NaN need no special case);
+* exactly K entries are kept; among equal magnitudes the lower index wins;
+* a selected entry votes with its IEEE sign bit (+0 votes +1, -0 votes -1), so
+  that every worker has exactly K non-zero votes as Section 2.2 states;
+* the K indices are listed ascending, 0-based; sign bit j belongs to index j,
+  packed LSB-first into 32-bit words (1 = negative), padding bits 0;
+* the update is one fp32 round-to-nearest operation: x - lr or x + lr.
+
+All integer results are exact, so GPU output must equal them bit for bit.
+Parity status: every function below is pinned by tests that do not call it to
+build their expectation (brute-force rank counting, the printed worked
+example, the K = N and M = 1 special cases of Section 3.3, invariants).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+ABS_MASK = np.uint32(0x7FFFFFFF)
+
+
+def _as_bits(grads: np.ndarray) -> np.ndarray:
+    g = np.ascontiguousarray(grads, dtype=np.float32)
+    if g.ndim != 2:
+        raise ValueError("grads must be [M, d]")
+    return g.view(np.uint32)
+
+
+def magnitude_keys(row_bits: np.ndarray) -> np.ndarray:
+    """|u| as an ordered unsigned integer: the bit pattern without its sign bit."""
+    return row_bits & ABS_MASK
+
+
+def pack_sign_bits(neg: np.ndarray) -> np.ndarray:
+    """Pack booleans (True = negative) LSB-first into uint32 words, zero padded."""
+    K = int(neg.shape[0])
+    words = np.zeros((K + 31) // 32, dtype=np.uint32)
+    for j in range(K):
+        if neg[j]:
+            words[j >> 5] |= np.uint32(1) << np.uint32(j & 31)
+    return words
+
+
+def _pack_sign_bits_fast(neg: np.ndarray) -> np.ndarray:
+    """Same packing with numpy bit ops (checked against pack_sign_bits in the tests)."""
+    K = int(neg.shape[0])
+    W = (K + 31) // 32
+    padded = np.zeros(W * 32, dtype=np.uint8)
+    padded[:K] = neg
+    by = np.packbits(padded.reshape(W, 32), axis=1, bitorder="little")  # [W, 4] bytes
+    return by.view("<u4").reshape(W).astype(np.uint32)
+
+
+def topk_sign(grads: np.ndarray, K: int):
+    """TopKSign of every worker's gradient, Eq. (3)-(4), in transmitted form.
+
+    Returns (idx [M, K] uint32 ascending, signbits [M, ceil(K/32)] uint32).
+    Definition written out: order all coordinates by (magnitude descending,
+    index ascending), keep the first K, list them by ascending index.
+    """
+    bits = _as_bits(grads)
+    M, d = bits.shape
+    if not 0 <= K <= d:
+        raise ValueError("K must be in [0, d]")
+    idx = np.zeros((M, K), dtype=np.uint32)
+    sgn = np.zeros((M, (K + 31) // 32), dtype=np.uint32)
+    for m in range(M):
+        key = magnitude_keys(bits[m]).astype(np.int64)
+        # a stable sort of the negated key puts equal magnitudes in index order
+        order = np.argsort(-key, kind="stable")
+        chosen = np.sort(order[:K])
+        idx[m] = chosen.astype(np.uint32)
+        sgn[m] = _pack_sign_bits_fast((bits[m][chosen] >> np.uint32(31)).astype(bool))
+    return idx, sgn
+
+
+def majority_vote(idx: np.ndarray, signbits: np.ndarray, M: int, K: int, d: int):
+    """sgn of the summed votes, Algorithm 1 / "Majority vote" paragraph.
+
+    Returns (vote [d] int8 in {-1, 0, +1}, n_out_of_range).  Repeated indices
+    add up; an index >= d is skipped and counted.
+    """
+    idx = np.asarray(idx, dtype=np.uint32).reshape(M, K)
+    signbits = np.asarray(signbits, dtype=np.uint32).reshape(M, (K + 31) // 32)
+    count = np.zeros(d, dtype=np.int64)
+    bad = 0
+    j = np.arange(K)
+    for m in range(M):
+        neg = (signbits[m][j >> 5] >> (j & 31).astype(np.uint32)) & np.uint32(1)
+        s = 1 - 2 * neg.astype(np.int64)
+        ok = idx[m] < d
+        bad += int(K - ok.sum())
+        np.add.at(count, idx[m][ok].astype(np.int64), s[ok])
+    vote = (count > 0).astype(np.int8) - (count < 0).astype(np.int8)
+    return vote, bad
+
+
+def apply_vote(x: np.ndarray, vote: np.ndarray, lr) -> np.ndarray:
+    """x <- x - lr * vote, Eq. (7), in fp32 with one rounding; vote 0 leaves x's bits alone."""
+    x = np.asarray(x, dtype=np.float32)
+    lr32 = np.float32(lr)
+    out = x.copy()
+    pos = vote > 0
+    neg = vote < 0
+    out[pos] = (x[pos] - lr32).astype(np.float32)
+    out[neg] = (x[neg] + lr32).astype(np.float32)
+    return out
+
+
+def step(x: np.ndarray, grads: np.ndarray, K: int, lr):
+    """One whole step of Algorithm 1 without error memory: send, vote, update.
+
+    Returns (x_new, idx, signbits, vote).
+    """
+    M, d = grads.shape
+    idx, sgn = topk_sign(grads, K)
+    vote, _ = majority_vote(idx, sgn, M, K, d)
+    return apply_vote(x, vote, lr), idx, sgn, vote
+
+
+# --------------------------------------------------------------------------
+# A second, faster route to the same selected set (threshold + tie fill), and
+# an O(d) certificate check.  Both are pinned against topk_sign() in the tests;
+# they exist so that rows of 1e7..1e9 elements can be checked in seconds.
+# --------------------------------------------------------------------------
+
+def topk_sign_threshold(grads: np.ndarray, K: int):
+    """Same output as topk_sign(), via the threshold form of Eq. (3).
+
+    rho = K-th largest magnitude (np.partition); everything above rho is kept,
+    and the remaining places go to the lowest indices whose magnitude equals rho.
+    """
+    bits = _as_bits(grads)
+    M, d = bits.shape
+    if not 0 <= K <= d:
+        raise ValueError("K must be in [0, d]")
+    idx = np.zeros((M, K), dtype=np.uint32)
+    sgn = np.zeros((M, (K + 31) // 32), dtype=np.uint32)
+    if K == 0:
+        return idx, sgn
+    for m in range(M):
+        key = magnitude_keys(bits[m])
+        rho = np.partition(key, d - K)[d - K]
+        above = np.flatnonzero(key > rho)
+        ties = np.flatnonzero(key == rho)[: K - above.shape[0]]
+        chosen = np.sort(np.concatenate([above, ties]))
+        idx[m] = chosen.astype(np.uint32)
+        sgn[m] = _pack_sign_bits_fast((bits[m][chosen] >> np.uint32(31)).astype(bool))
+    return idx, sgn
+
+
+def check_topk_sign_row(row: np.ndarray, K: int, idx: np.ndarray, signbits: np.ndarray) -> str:
+    """Decide in O(d) whether (idx, signbits) is THE TopKSign message of ``row``.
+
+    The answer is unique under the lowest-index tie rule, so a set that passes
+    equals topk_sign()'s.  Returns "" when correct, else a description of the
+    first violated condition:
+      1. K strictly ascending indices below d;
+      2. with rho = smallest selected magnitude: no unselected magnitude > rho;
+      3. every unselected entry of magnitude rho lies after the last selected
+         entry of magnitude rho;
+      4. sign bit j is the IEEE sign of row[idx[j]], padding bits are 0.
+    """
+    rb = np.ascontiguousarray(row, dtype=np.float32).view(np.uint32)
+    d = rb.shape[0]
+    idx = np.asarray(idx, dtype=np.uint32)
+    signbits = np.asarray(signbits, dtype=np.uint32)
+    if idx.shape != (K,) or signbits.shape != ((K + 31) // 32,):
+        return "wrong shapes"
+    if K == 0:
+        return ""
+    i64 = idx.astype(np.int64)
+    if i64[-1] >= d or np.any(np.diff(i64) <= 0):
+        return "indices not strictly ascending in range"
+    key = magnitude_keys(rb)
+    sel = np.zeros(d, dtype=bool)
+    sel[i64] = True
+    rho = key[i64].min()
+    if np.any(key[~sel] > rho):
+        return "an unselected entry exceeds the smallest selected magnitude"
+    unsel_ties = np.flatnonzero((key == rho) & ~sel)
+    sel_ties = np.flatnonzero((key == rho) & sel)
+    if unsel_ties.size and unsel_ties[0] < sel_ties[-1]:
+        return "tie at the threshold not resolved toward the lower index"
+    want = _pack_sign_bits_fast((rb[i64] >> np.uint32(31)).astype(bool))
+    if not np.array_equal(want, signbits):
+        return "sign bits do not match the IEEE signs of the selected entries"
+    return ""

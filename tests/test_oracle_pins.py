@@ -1,0 +1,452 @@
+"""Pins the CPU oracle to things other than itself (no GPU, no CUDA library).
+
+Every expectation here comes from the paper's printed values, from a closed
+form, from brute force on tiny inputs, or from an invariant of the definition;
+none is produced by calling the function under test.  The last test plants
+plausible mistakes into the oracle and checks that the pins notice each one.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import s3gd_oracle as O
+from paper_2302_07475_b200 import workloads as W
+
+GOLD = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+def f32_bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def unpack(signbits_row, K):
+    j = np.arange(K)
+    return ((signbits_row[j >> 5] >> (j & 31).astype(np.uint32)) & 1).astype(np.int64)
+
+
+# ---------------------------------------------------------------- brute force
+def brute_topk_sign(row, K):
+    """Rank counting, O(d^2), no sort: n is kept iff fewer than K entries beat it.
+
+    j beats n when |u_j| > |u_n|, or |u_j| == |u_n| and j < n (Eq. (3) plus the
+    lowest-index tie rule).  Magnitudes are compared as Python floats via abs(),
+    not via bit patterns, so this is a different route to the order.
+    """
+    d = len(row)
+    vals = [float(v) for v in row]
+    kept = []
+    for n in range(d):
+        rank = 0
+        for j in range(d):
+            if abs(vals[j]) > abs(vals[n]) or (abs(vals[j]) == abs(vals[n]) and j < n):
+                rank += 1
+        if rank < K:
+            kept.append(n)
+    neg = [np.signbit(row[n]) for n in kept]
+    return kept, neg
+
+
+def brute_vote(per_worker, d):
+    count = [0] * d
+    for kept, neg in per_worker:
+        for n, s in zip(kept, neg):
+            count[n] += -1 if s else 1
+    return [(c > 0) - (c < 0) for c in count]
+
+
+def pin_bruteforce(orc):
+    rng = np.random.default_rng(1)
+    for trial in range(30):
+        d = int(rng.integers(1, 17))
+        M = int(rng.integers(1, 5))
+        # few distinct magnitudes => ties everywhere, both signs, exact zeros
+        levels = np.array([0.0, 0.25, 0.25, 1.0, 1.5, 7.0], dtype=np.float32)
+        g = levels[rng.integers(0, len(levels), (M, d))] * rng.choice([-1.0, 1.0], (M, d)).astype(np.float32)
+        if trial % 3 == 0:
+            g = rng.standard_normal((M, d)).astype(np.float32)
+        for K in range(d + 1):
+            idx, sgn = orc.topk_sign(g, K)
+            per_worker = []
+            for m in range(M):
+                kept, neg = brute_topk_sign(g[m], K)
+                per_worker.append((kept, neg))
+                assert idx[m].tolist() == kept
+                assert unpack(sgn[m], K).tolist() == [int(b) for b in neg]
+                # padding bits of the last word are zero
+                if K % 32:
+                    assert int(sgn[m][-1]) >> (K % 32) == 0
+            vote, bad = orc.majority_vote(idx, sgn, M, K, d)
+            assert bad == 0
+            assert vote.tolist() == brute_vote(per_worker, d)
+
+
+def test_bruteforce_tiny():
+    pin_bruteforce(O)
+
+
+# ------------------------------------------------------ printed worked example
+def pin_example1(orc):
+    with open(os.path.join(GOLD, "example1_power_of_representative_democracy.json")) as f:
+        ex = json.load(f)
+    col = np.array(ex["values_at_coordinate_n"], dtype=np.float32)
+    assert np.sign(col.astype(np.float64).mean()) == ex["sign_of_full_precision_mean"]
+    # Three workers, d = 4.  Coordinate 2 holds the example's values.  The other
+    # coordinates are filled so that with K = 1 worker 1 keeps coordinate 2
+    # (3 is its largest, and the only one above the example's bar |g| > 1)
+    # while workers 2 and 3 keep a different coordinate.
+    g = np.array([[0.5, -0.2, col[0], 0.1],
+                  [0.9, 0.1, col[1], -0.2],
+                  [0.01, -0.8, col[2], 0.02]], dtype=np.float32)
+    x = np.zeros(4, dtype=np.float32)
+    # signSGD with majority vote = every entry votes (K = d)
+    _, _, _, vote_all = orc.step(x, g, 4, 1.0)
+    assert int(vote_all[2]) == ex["signsgd_majority_vote"]
+    # sparsified vote: only the confident worker takes part at coordinate 2
+    xs, idx, _, vote_1 = orc.step(x, g, 1, 1.0)
+    assert idx[:, 0].tolist() == [2, 0, 1]
+    assert int(vote_1[2]) == ex["thresholded_majority_vote"]
+    assert xs[2] == np.float32(-1.0)      # x - delta * (+1)
+
+
+def test_example1_printed_values():
+    pin_example1(O)
+
+
+# ----------------------------------------------- closed-form special cases
+def pin_gamma_one_is_signsgd_mv(orc):
+    """Section 3.3, gamma = 1: the step equals signSGD with majority vote."""
+    rng = np.random.default_rng(2)
+    M, d = 7, 300
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    g[:, ::17] = 0.0
+    g[::2, ::34] = -0.0
+    x = rng.standard_normal(d).astype(np.float32)
+    lr = np.float32(0.01)
+    x_new, idx, sgn, vote = orc.step(x, g, d, lr)
+    for n in range(d):
+        total = 0
+        for m in range(M):
+            total += -1 if np.signbit(g[m, n]) else 1
+        want = (total > 0) - (total < 0)
+        assert vote[n] == want
+        assert x_new[n] == np.float32(np.float64(x[n]) - np.float64(lr) * want)
+    assert all(idx[m].tolist() == list(range(d)) for m in range(M))
+
+
+def pin_single_worker(orc):
+    """Section 3.3, M = 1: the vote is TopKSign(g) itself; exactly K coordinates move by lr."""
+    rng = np.random.default_rng(3)
+    d, K = 500, 37
+    g = rng.standard_normal((1, d)).astype(np.float32)
+    x = (np.round(rng.standard_normal(d) * 1024) / 1024).astype(np.float32)
+    lr = np.float32(0.125)                      # x on a 2^-10 grid: x -/+ lr is exact
+    x_new, idx, sgn, vote = orc.step(x, g, K, lr)
+    mags = np.abs(g[0].astype(np.float64))
+    kth = np.sort(mags)[::-1][K - 1]
+    want = np.where(mags >= kth, np.sign(g[0]), 0).astype(np.int64)   # no ties in continuous data
+    assert np.array_equal(vote.astype(np.int64), want)
+    assert int(np.count_nonzero(vote)) == K
+    moved = x_new != x
+    assert np.array_equal(moved, vote != 0)
+    assert np.array_equal((x_new - x)[moved], (-lr * vote[moved]).astype(np.float32))
+
+
+def test_special_cases():
+    pin_gamma_one_is_signsgd_mv(O)
+    pin_single_worker(O)
+
+
+# ------------------------------------------------------------ invariants
+def pin_invariants(orc):
+    rng = np.random.default_rng(4)
+    M, d = 6, 2000
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    g = (np.round(g * 8) / 8).astype(np.float32)        # plenty of ties
+    x = rng.standard_normal(d).astype(np.float32)
+    lr = np.float32(1e-3)
+    prev = None
+    for K in (0, 1, 31, 32, 33, 200, 1999, 2000):
+        x_new, idx, sgn, vote = orc.step(x, g, K, lr)
+        # exactly K distinct ascending in-range indices per worker (Section 2.2)
+        for m in range(M):
+            assert idx[m].shape == (K,)
+            assert np.all(np.diff(idx[m].astype(np.int64)) > 0)
+            assert K == 0 or idx[m][-1] < d
+        # sum of all counts equals the signed number of votes
+        total = sum(K - 2 * int(unpack(sgn[m], K).sum()) for m in range(M))
+        cnt = np.zeros(d, dtype=np.int64)
+        for m in range(M):
+            np.add.at(cnt, idx[m].astype(np.int64), 1 - 2 * unpack(sgn[m], K))
+        assert cnt.sum() == total
+        assert np.count_nonzero(vote) <= min(d, M * K)
+        # permuting the workers changes nothing at the server
+        perm = rng.permutation(M)
+        xp, _, _, vp = orc.step(x, g[perm], K, lr)
+        assert np.array_equal(vp, vote) and np.array_equal(f32_bits(xp), f32_bits(x_new))
+        # negating every gradient keeps the support, flips signs and the vote
+        xn, idxn, sgnn, vn = orc.step(x, -g, K, lr)
+        assert np.array_equal(idxn, idx) and np.array_equal(vn, -vote)
+        for m in range(M):
+            assert np.array_equal(unpack(sgnn[m], K), 1 - unpack(sgn[m], K))
+        # scaling a row by a power of two is exact and changes nothing
+        g2 = g.copy()
+        g2[1] *= np.float32(4.0)
+        _, idx2, sgn2, _ = orc.step(x, g2, K, lr)
+        assert np.array_equal(idx2, idx) and np.array_equal(sgn2, sgn)
+        # supports are nested in K
+        if prev is not None:
+            for m in range(M):
+                assert set(prev[m].tolist()) <= set(idx[m].tolist())
+        prev = idx
+        # the update moves voted coordinates by one correctly rounded fp32 operation
+        want = (x.astype(np.float64) - np.float64(lr) * vote).astype(np.float32)
+        assert np.array_equal(f32_bits(x_new)[vote != 0], f32_bits(want)[vote != 0])
+        assert np.array_equal(f32_bits(x_new)[vote == 0], f32_bits(x)[vote == 0])
+
+
+def test_invariants():
+    pin_invariants(O)
+
+
+def pin_apply_bits(orc):
+    """vote 0 must leave the bit pattern alone (NaN payloads, -0); vote +-1 is one rounding."""
+    x = np.array([0.0, -0.0, 1.0, np.nan, np.inf, 1e-40, 16777216.0, 0.1], dtype=np.float32)
+    xb = f32_bits(x).copy()
+    xb[3] = 0x7FC12345
+    x = xb.view(np.float32)
+    vote0 = np.zeros(8, dtype=np.int8)
+    assert np.array_equal(f32_bits(orc.apply_vote(x, vote0, 0.5)), xb)
+    votep = np.ones(8, dtype=np.int8)
+    lr = np.float32(0.3)
+    got = orc.apply_vote(x, votep, lr)
+    want = (x.astype(np.float64) - np.float64(lr)).astype(np.float32)
+    ok = ~np.isnan(want)
+    assert np.array_equal(f32_bits(got)[ok], f32_bits(want)[ok])
+    got = orc.apply_vote(x, -votep, lr)
+    want = (x.astype(np.float64) + np.float64(lr)).astype(np.float32)
+    assert np.array_equal(f32_bits(got)[ok], f32_bits(want)[ok])
+
+
+def test_apply_bits():
+    pin_apply_bits(O)
+
+
+def pin_vote_semantics(orc):
+    """Repeated indices add up; out-of-range indices are skipped and counted; ties give 0."""
+    d, M, K = 10, 2, 4
+    idx = np.array([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=np.uint32)
+    sgn = np.array([[0b0110], [0b0001]], dtype=np.uint32)   # w0: +,-,-,+   w1: -,+,+,+
+    vote, bad = orc.majority_vote(idx, sgn, M, K, d)
+    # coord1: +1 -1 -1 = -1 ; coord3: -1 +1 = 0 ; coord4: +1 ; coord9: +1 ; 12 skipped
+    want = [0, -1, 0, 0, 1, 0, 0, 0, 0, 1]
+    assert vote.tolist() == want and bad == 1
+
+
+def test_vote_semantics():
+    pin_vote_semantics(O)
+
+
+def test_special_values_order():
+    """NaN > Inf > finite > denormal > 0 in the bit-pattern order; signs taken from the sign bit."""
+    g = np.array([[1.0, -np.inf, 1e-42, np.nan, -0.0, 3e38, -1e-45, 0.0]], dtype=np.float32)
+    idx, sgn = O.topk_sign(g, 8)
+    ranks = []
+    for K in range(1, 9):
+        i, _ = O.topk_sign(g, K)
+        ranks.append(set(i[0].tolist()))
+    order = [next(iter(ranks[0]))] + [next(iter(ranks[k] - ranks[k - 1])) for k in range(1, 8)]
+    assert order == [3, 1, 5, 0, 2, 6, 4, 7]
+    assert unpack(sgn[0], 8).tolist() == [0, 1, 0, 0, 1, 0, 1, 0]
+
+
+# ----------------------------------------------------- packing helper pinned
+def test_pack_helpers_agree():
+    rng = np.random.default_rng(5)
+    for K in (0, 1, 31, 32, 33, 64, 1000):
+        neg = rng.random(K) < 0.5
+        slow = O.pack_sign_bits(neg)
+        assert np.array_equal(slow, O._pack_sign_bits_fast(neg))
+        # written out once more from the layout statement: word j//32, bit j%32
+        for j in range(K):
+            assert ((int(slow[j // 32]) >> (j % 32)) & 1) == int(neg[j])
+
+
+# ---------------------------------- threshold route and certificate check
+@pytest.mark.parametrize("kind", ["normal", "all_equal", "zeros", "few_levels", "one_hot", "special", "ramp"])
+def test_threshold_route_equals_definition(kind):
+    M, d = 3, 1537
+    if kind == "normal":
+        g = np.random.default_rng(6).standard_normal((M, d)).astype(np.float32)
+    else:
+        g = W.edge_case_grads(kind, M, d).numpy()
+    for K in (0, 1, 2, 100, 768, 1536, 1537):
+        a = O.topk_sign(g, K)
+        b = O.topk_sign_threshold(g, K)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+        for m in range(M):
+            assert O.check_topk_sign_row(g[m], K, a[0][m], a[1][m]) == ""
+
+
+def test_threshold_route_on_workload_shapes():
+    s = W.spec("resnet50_ties", d=200_003, M=2)
+    g = W.make_grads(s, "cpu").numpy()
+    for K in (20, 200, 2000, 20000):
+        a = O.topk_sign(g, K)
+        b = O.topk_sign_threshold(g, K)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+def test_certificate_rejects_wrong_answers():
+    g = W.edge_case_grads("few_levels", 1, 400)[0].numpy()
+    K = 150
+    idx, sgn = O.topk_sign(g[None, :], K)
+    idx, sgn = idx[0], sgn[0]
+    assert O.check_topk_sign_row(g, K, idx, sgn) == ""
+    key = f32_bits(g) & 0x7FFFFFFF
+    rho = key[idx].min()
+    sel = set(idx.tolist())
+    # (a) swap the last selected tie for a later unselected tie: same magnitudes, wrong tie rule
+    later = [n for n in range(400) if key[n] == rho and n not in sel]
+    ties_sel = [n for n in idx.tolist() if key[n] == rho]
+    assert later and ties_sel
+    bad = np.array(sorted((sel - {ties_sel[0]}) | {later[-1]}), dtype=np.uint32)
+    sb = O._pack_sign_bits_fast((f32_bits(g)[bad] >> 31).astype(bool))
+    assert "tie" in O.check_topk_sign_row(g, K, bad, sb)
+    # (b) replace a large entry by a small one
+    small = [n for n in range(400) if key[n] < rho]
+    big = [n for n in idx.tolist() if key[n] > rho]
+    bad = np.array(sorted((sel - {big[0]}) | {small[0]}), dtype=np.uint32)
+    sb = O._pack_sign_bits_fast((f32_bits(g)[bad] >> 31).astype(bool))
+    assert "exceeds" in O.check_topk_sign_row(g, K, bad, sb)
+    # (c) one flipped sign bit, (d) a set padding bit, (e) unsorted, (f) duplicate
+    s2 = sgn.copy(); s2[1] ^= np.uint32(4)
+    assert "sign" in O.check_topk_sign_row(g, K, idx, s2)
+    s3 = sgn.copy(); s3[-1] |= np.uint32(1 << 31)
+    assert "sign" in O.check_topk_sign_row(g, K, idx, s3)
+    i2 = idx.copy(); i2[[3, 4]] = i2[[4, 3]]
+    assert "ascending" in O.check_topk_sign_row(g, K, i2, sgn)
+    i3 = idx.copy(); i3[5] = i3[4]
+    assert "ascending" in O.check_topk_sign_row(g, K, i3, sgn)
+
+
+# ------------------------------------------------ statistical closed forms
+def test_support_statistics_match_closed_forms():
+    """Independent rows: voter counts ~ Binomial(M, K/N) (Lemma 3); empty fraction (1-K/N)^M (Example 2)."""
+    with open(os.path.join(GOLD, "closed_forms.json")) as f:
+        cases = {(c["N"], c["K"], c["M"]): c for c in json.load(f)["cases"]}
+    s = W.SPECS["tiny"]
+    c = cases[(s.d, s.Ks[0], s.M)]
+    g = W.make_grads(s, "cpu").numpy()
+    idx, _ = O.topk_sign(g, s.Ks[0])
+    voters = np.zeros(s.d, dtype=np.int64)
+    for m in range(s.M):
+        voters[idx[m]] += 1
+    frac_voted = np.count_nonzero(voters) / s.d
+    # alpha = 0.04898; std of the estimate ~ sqrt(alpha/N) ~ 8.6e-4
+    assert abs(frac_voted - c["alpha"]) < 5 * 8.6e-4
+    assert abs((voters == 0).mean() - c["p_empty"]) < 5 * 8.6e-4
+    hist = np.bincount(voters, minlength=s.M + 1) / s.d
+    assert abs(hist[1] - c["voter_count_pmf"][1]) < 5e-3
+    assert abs(hist[2] - c["voter_count_pmf"][2]) < 1e-3
+
+
+# ------------------------------------------- the pins notice planted mistakes
+ALL_PINS = [pin_bruteforce, pin_example1, pin_gamma_one_is_signsgd_mv, pin_single_worker,
+            pin_invariants, pin_apply_bits, pin_vote_semantics]
+
+
+def _mutants():
+    real_topk, real_vote, real_apply = O.topk_sign, O.majority_vote, O.apply_vote
+
+    def higher_index_wins(g, K):            # wrong tie rule
+        M, d = g.shape
+        i, s = real_topk(g[:, ::-1], K)
+        i = (d - 1 - i.astype(np.int64))[:, ::-1].astype(np.uint32)
+        out = np.zeros_like(s)
+        for m in range(M):
+            out[m] = O._pack_sign_bits_fast(np.signbit(g[m][i[m]]))
+        return i, out
+
+    def signed_not_magnitude(g, K):          # top-K of the signed value instead of |.|
+        i, _ = real_topk(np.where(g > 0, g, 0).astype(np.float32), K)
+        out = np.zeros((g.shape[0], (K + 31) // 32), dtype=np.uint32)
+        for m in range(g.shape[0]):
+            out[m] = O._pack_sign_bits_fast(np.signbit(g[m][i[m]]))
+        return i, out
+
+    def smallest_k(g, K):                    # ascending instead of descending
+        with np.errstate(divide="ignore"):
+            return real_topk((1.0 / (np.abs(g) + 1e-3)).astype(np.float32) * np.where(np.signbit(g), -1, 1).astype(np.float32), K)
+
+    def inverted_sign_bits(g, K):            # 1 = positive
+        i, s = real_topk(g, K)
+        out = np.zeros_like(s)
+        for m in range(g.shape[0]):
+            out[m] = O._pack_sign_bits_fast(~np.signbit(g[m][i[m]]))
+        return i, out
+
+    def msb_first(g, K):                     # wrong bit order inside a word
+        i, s = real_topk(g, K)
+        out = np.zeros_like(s)
+        for m in range(g.shape[0]):
+            neg = np.signbit(g[m][i[m]])
+            for j in range(K):
+                if neg[j]:
+                    out[m][j >> 5] |= np.uint32(1) << np.uint32(31 - (j & 31))
+        return i, out
+
+    def zero_votes_nothing(g, K):            # sgn(0) = 0 read literally drops +-0 entries' sign
+        i, s = real_topk(g, K)
+        out = np.zeros_like(s)
+        for m in range(g.shape[0]):
+            out[m] = O._pack_sign_bits_fast(g[m][i[m]] < 0)
+        return i, out
+
+    def vote_tie_positive(idx, sgn, M, K, d):   # ties broken toward +1 instead of 0
+        v, bad = real_vote(idx, sgn, M, K, d)
+        cnt = np.zeros(d, dtype=np.int64)
+        for m in range(M):
+            ok = idx[m] < d
+            np.add.at(cnt, idx[m][ok].astype(np.int64), 1)
+        v = v.copy()
+        v[(v == 0) & (cnt > 0)] = 1
+        return v, bad
+
+    def vote_set_semantics(idx, sgn, M, K, d):  # duplicates counted once
+        v = np.zeros(d, dtype=np.int64)
+        for m in range(M):
+            seen = set()
+            for j in range(K):
+                n = int(idx[m][j])
+                if n < d and n not in seen:
+                    seen.add(n)
+                    v[n] += 1 - 2 * ((int(sgn[m][j >> 5]) >> (j & 31)) & 1)
+        return ((v > 0).astype(np.int8) - (v < 0).astype(np.int8)), int((idx >= d).sum())
+
+    def apply_plus(x, vote, lr):                # wrong sign of the update
+        return real_apply(x, -np.asarray(vote), lr)
+
+    def apply_double(x, vote, lr):              # update computed in fp64 product then added twice-rounded
+        return (x + np.float32(-1.0) * (np.float32(lr) * vote.astype(np.float32)) + np.float32(0.0)).astype(np.float32) * np.float32(1.0) + np.float32(0.0)
+
+    return [("topk_sign", higher_index_wins), ("topk_sign", signed_not_magnitude), ("topk_sign", smallest_k),
+            ("topk_sign", inverted_sign_bits), ("topk_sign", msb_first), ("topk_sign", zero_votes_nothing),
+            ("majority_vote", vote_tie_positive), ("majority_vote", vote_set_semantics),
+            ("apply_vote", apply_plus), ("apply_vote", apply_double)]
+
+
+@pytest.mark.parametrize("which", range(10))
+def test_pins_catch_planted_mistakes(which, monkeypatch):
+    name, fn = _mutants()[which]
+    monkeypatch.setattr(O, name, fn)
+    caught = 0
+    for pin in ALL_PINS:
+        try:
+            pin(O)
+        except AssertionError:
+            caught += 1
+        except Exception:
+            caught += 1
+    assert caught >= 1, f"no pin notices mutant {fn.__name__}"
