@@ -1,0 +1,155 @@
+/*
+ * s3gd.h -- C ABI of the S3GD-MV compression / aggregation / update step for
+ * one NVIDIA B200 (sm_100a).
+ *
+ * The operations are those of Park & Lee, "Sparse-SignSGD with Majority Vote
+ * for Communication-Efficient Distributed Learning" (arXiv 2302.07475):
+ * M workers each hold a gradient of length d (the paper's N); each sends the
+ * signs of its K largest-magnitude entries (TopKSign, Section 2.1 Eq. (3)-(4)),
+ * the server takes the sign of the summed votes (Section 2.2 "Majority vote",
+ * Algorithm 1) and every worker moves x by -lr times that sign vector
+ * (Section 2.2 Eq. (7)).  Here the M workers are the rows of one gradient
+ * buffer in device memory and the "network" is device memory.
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - "dev" pointers are device pointers valid on the current CUDA device;
+ *    "host" means ordinary host memory.  The library never allocates, frees or
+ *    retains a pointer.  Every buffer, including the workspace, is the caller's.
+ *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *    the default stream).  No call synchronises except s3gd_device_status().
+ *  - Magnitude order is the unsigned order of the fp32 bit pattern with the sign
+ *    bit cleared.  Denormals are not flushed; NaN and Inf order by bit pattern.
+ *  - Exactly K entries are kept per worker; equal magnitudes go to the lower
+ *    index.  A kept entry votes with its IEEE sign bit (+0 votes +1, -0 votes -1).
+ *  - Indices are 0-based uint32 and ascending within a worker.  Sign bit j of a
+ *    worker belongs to its j-th index: word j/32, bit j%32 (LSB first),
+ *    1 = negative; unused bits of the last word are 0.
+ *  - Return value: S3GD_OK or an error detected on the host BEFORE anything is
+ *    enqueued (outputs untouched).  Conditions only the device can see are
+ *    recorded in the workspace and read back with s3gd_device_status().
+ */
+#ifndef S3GD_H_
+#define S3GD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define S3GD_API __attribute__((visibility("default")))
+#else
+#define S3GD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum s3gd_status {
+  S3GD_OK = 0,
+  S3GD_ERR_INVALID_ARG = 1, /* NULL pointer, M <= 0, d == 0, d >= 2^32, K > d, bad alignment */
+  S3GD_ERR_WORKSPACE = 2,   /* workspace NULL, smaller than s3gd_workspace_bytes(), or not 256-byte aligned */
+  S3GD_ERR_CUDA = 3,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
+  S3GD_ERR_INDEX_RANGE = 4, /* device: an index >= d was given to s3gd_majority_vote (skipped) */
+  S3GD_ERR_INTERNAL = 5     /* device: a selection did not produce exactly K entries */
+} s3gd_status;
+
+/* Human-readable name of a status code.  Host.  Never NULL. */
+S3GD_API const char* s3gd_status_string(s3gd_status st);
+
+/*
+ * Bytes of device workspace that the calls below need for (M, d, K).  Host, pure.
+ * A workspace sized for (M, d, K) is only guaranteed to serve calls with exactly
+ * these three values.  Returns 0 for invalid arguments.  The workspace must be
+ * 256-byte aligned.  Its contents need not be initialised and are not preserved.
+ */
+S3GD_API size_t s3gd_workspace_bytes(int M, uint64_t d, uint64_t K);
+
+/*
+ * TopKSign of every worker's gradient in transmitted form
+ * (Section 2.1, Eq. (3)-(4); Section 2.2 "Gradient compression").
+ *
+ *  grads        dev, const  [M x d] fp32 row-major (row m = worker m), 4-byte aligned
+ *  out_idx      dev         [M x K] uint32, ascending per row
+ *  out_signbits dev         [M x ceil(K/32)] uint32
+ *  ws, ws_bytes dev         workspace, >= s3gd_workspace_bytes(M, d, K)
+ *
+ * K == 0 is valid and writes nothing.  K == d keeps everything.
+ */
+S3GD_API s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K,
+                           uint32_t* out_idx, uint32_t* out_signbits,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Majority vote at the server (Section 2.2 "Majority vote"; Algorithm 1):
+ * out_vote[n] = sgn( sum over workers and their entries j with idx == n of
+ * (1 - 2 * signbit_j) ), so a coordinate nobody sent, or an exact tie, gets 0.
+ *
+ *  idx       dev, const  [M x K] uint32 (any order; repeated indices add up;
+ *                        an index >= d is skipped and S3GD_ERR_INDEX_RANGE is recorded)
+ *  signbits  dev, const  [M x ceil(K/32)] uint32
+ *  out_vote  dev         [d] int8 in {-1, 0, +1}
+ *  ws        dev         workspace, >= s3gd_workspace_bytes(M, d, K); holds the int32 counters
+ */
+S3GD_API s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K,
+                               uint64_t d, int8_t* out_vote,
+                               void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Model update (Section 2.2, Eq. (7)): x[n] <- fl32(x[n] - lr * vote[n]), one
+ * round-to-nearest fp32 operation; where vote[n] == 0 the bits of x[n] are left alone.
+ *
+ *  x     dev  [d] fp32, updated in place
+ *  vote  dev, const [d] int8; any positive value counts as +1, any negative as -1
+ */
+S3GD_API s3gd_status s3gd_apply(float* x, const int8_t* vote, uint64_t d, float lr, void* stream);
+
+/*
+ * One whole step of Algorithm 1 after the local gradients exist (its "send",
+ * "receive" and "x <-" lines): TopKSign per worker, majority vote, update of x.
+ * Produces exactly what s3gd_topk_sign -> s3gd_majority_vote -> s3gd_apply
+ * produce, without writing the intermediate message unless asked to.
+ * With K == d this is signSGD with majority vote (Section 3.3, gamma = 1) and
+ * runs as one streaming pass over the M sign planes.
+ *
+ *  x            dev  [d] fp32, updated in place
+ *  grads        dev, const [M x d]
+ *  opt_idx      dev or NULL  [M x K]            (as s3gd_topk_sign)
+ *  opt_signbits dev or NULL  [M x ceil(K/32)]   (must be given together with opt_idx)
+ *  opt_vote     dev or NULL  [d] int8
+ */
+S3GD_API s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr,
+                      uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Waits for `stream`, then reports what the kernels of earlier calls on this
+ * workspace recorded: S3GD_OK, S3GD_ERR_INDEX_RANGE or S3GD_ERR_INTERNAL.
+ * The record is cleared by the next s3gd_topk_sign / s3gd_majority_vote / s3gd_step.
+ * If info is not NULL (host, 8 x uint32) it receives diagnostic counters:
+ *   [0] status word  [1] rows that took the exact multi-pass route
+ *   [2] out-of-range indices skipped  [3] rows whose selection size != K
+ *   [4] largest candidate count of a row  [5..7] reserved (0)
+ */
+S3GD_API s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* info);
+
+/*
+ * Measurement aid (the paper reports no timings; this has no counterpart there).
+ * Between s3gd_profile_begin(max_steps) and s3gd_profile_end(), every s3gd_step call of
+ * this process records CUDA events on its stream at its phase boundaries, for at most
+ * max_steps calls.  s3gd_profile_end synchronises the device and writes, for each recorded
+ * call, 5 durations in milliseconds to out_ms (host, [max_steps x 5], may be NULL):
+ *   [0] clear counters + sampled threshold   [1] filter pass over the gradients
+ *   [2] radix passes for the exact threshold [3] per-tile counts, scan, ordered emission
+ *   [4] sign of the counters + update of x   (K == d: [4] is the whole sign-plane pass)
+ * *n_steps (host) receives the number of recorded calls and *launches (host) the number
+ * of kernels this library enqueued since s3gd_profile_begin.  Not thread-safe; one
+ * profiling session at a time.  The events are created and destroyed by these two calls.
+ */
+S3GD_API s3gd_status s3gd_profile_begin(int max_steps);
+S3GD_API s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S3GD_H_ */

@@ -1,0 +1,11 @@
+"""S3GD-MV step (top-K sign compression, majority vote, update) for NVIDIA B200.
+
+The compute path is the CUDA library ``libs3gd.so`` (sources in ``csrc/``, C ABI in
+``include/s3gd.h``); ``binding`` marshals torch tensors into it.  ``workloads``
+draws the seeded synthetic gradient batches used by tests and benchmarks.
+"""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    S3gdError, alloc_workspace, load, s3gd_apply, s3gd_device_status, s3gd_majority_vote,
+    s3gd_profile_begin, s3gd_profile_end, s3gd_status_string, s3gd_step, s3gd_topk_sign, s3gd_workspace_bytes,
+)

@@ -1,0 +1,183 @@
+"""ctypes binding of libs3gd.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the CUDA kernels of the library; nothing here
+computes.  torch is used for device buffers and the current stream.  If the
+library is missing or a tensor is not a contiguous CUDA tensor of the right
+dtype the call raises -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libs3gd.so")
+
+S3GD_OK = 0
+STATUS_NAMES = {
+    0: "S3GD_OK", 1: "S3GD_ERR_INVALID_ARG", 2: "S3GD_ERR_WORKSPACE", 3: "S3GD_ERR_CUDA",
+    4: "S3GD_ERR_INDEX_RANGE", 5: "S3GD_ERR_INTERNAL",
+}
+
+EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
+           "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end")
+
+
+class S3gdError(RuntimeError):
+    def __init__(self, call: str, code: int):
+        super().__init__(f"{call} returned {STATUS_NAMES.get(code, code)}")
+        self.code = code
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load the shared library (once) and declare the argument types of every export."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(
+            f"{p} not found: build it with `python -m paper_2302_07475_b200.build` (needs nvcc); "
+            "there is no fallback implementation")
+    lib = ctypes.CDLL(p)
+    vp, u64, u32p, sz = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_size_t
+    lib.s3gd_status_string.restype = ctypes.c_char_p
+    lib.s3gd_status_string.argtypes = [ctypes.c_int]
+    lib.s3gd_workspace_bytes.restype = sz
+    lib.s3gd_workspace_bytes.argtypes = [ctypes.c_int, u64, u64]
+    lib.s3gd_topk_sign.restype = ctypes.c_int
+    lib.s3gd_topk_sign.argtypes = [vp, ctypes.c_int, u64, u64, u32p, u32p, vp, sz, vp]
+    lib.s3gd_majority_vote.restype = ctypes.c_int
+    lib.s3gd_majority_vote.argtypes = [u32p, u32p, ctypes.c_int, u64, u64, vp, vp, sz, vp]
+    lib.s3gd_apply.restype = ctypes.c_int
+    lib.s3gd_apply.argtypes = [vp, vp, u64, ctypes.c_float, vp]
+    lib.s3gd_step.restype = ctypes.c_int
+    lib.s3gd_step.argtypes = [vp, vp, ctypes.c_int, u64, u64, ctypes.c_float, u32p, u32p, vp, vp, sz, vp]
+    lib.s3gd_device_status.restype = ctypes.c_int
+    lib.s3gd_device_status.argtypes = [vp, vp, ctypes.c_void_p]
+    lib.s3gd_profile_begin.restype = ctypes.c_int
+    lib.s3gd_profile_begin.argtypes = [ctypes.c_int]
+    lib.s3gd_profile_end.restype = ctypes.c_int
+    lib.s3gd_profile_end.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, numel: Optional[int] = None, name: str = "tensor"):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+    if numel is not None and t.numel() < numel:
+        raise ValueError(f"{name} has {t.numel()} elements, needs {numel}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(t: torch.Tensor):
+    return ctypes.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def _check(call: str, code: int) -> None:
+    if code != S3GD_OK:
+        raise S3gdError(call, code)
+
+
+def s3gd_status_string(code: int) -> str:
+    return load().s3gd_status_string(int(code)).decode()
+
+
+def s3gd_workspace_bytes(M: int, d: int, K: int) -> int:
+    return int(load().s3gd_workspace_bytes(int(M), int(d), int(K)))
+
+
+def alloc_workspace(M: int, d: int, K: int, device="cuda") -> torch.Tensor:
+    """A uint8 CUDA tensor of s3gd_workspace_bytes(M, d, K) bytes (torch allocations are 512-byte aligned)."""
+    n = s3gd_workspace_bytes(M, d, K)
+    if n == 0:
+        raise ValueError("invalid (M, d, K)")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def words(K: int) -> int:
+    return (int(K) + 31) // 32
+
+
+def s3gd_topk_sign(grads: torch.Tensor, K: int, out_idx: torch.Tensor, out_signbits: torch.Tensor,
+                   ws: torch.Tensor) -> None:
+    """grads [M, d] fp32 -> out_idx [M, K] (uint32 values in int32 storage), out_signbits [M, ceil(K/32)]."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (g, M, d, K, _ptr(out_idx, torch.int32, M * K, "out_idx"),
+            _ptr(out_signbits, torch.int32, M * words(K), "out_signbits"),
+            _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(grads.device):
+        code = load().s3gd_topk_sign(*args, _stream(grads))
+    _check("s3gd_topk_sign", code)
+
+
+def s3gd_majority_vote(idx: torch.Tensor, signbits: torch.Tensor, M: int, K: int, d: int,
+                       out_vote: torch.Tensor, ws: torch.Tensor) -> None:
+    """idx [M, K], signbits [M, ceil(K/32)] -> out_vote [d] int8 in {-1, 0, +1}."""
+    args = (_ptr(idx, torch.int32, M * K, "idx"), _ptr(signbits, torch.int32, M * words(K), "signbits"), M, K, d,
+            _ptr(out_vote, torch.int8, d, "out_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(out_vote.device):
+        code = load().s3gd_majority_vote(*args, _stream(out_vote))
+    _check("s3gd_majority_vote", code)
+
+
+def s3gd_apply(x: torch.Tensor, vote: torch.Tensor, lr: float) -> None:
+    """x [d] fp32 updated in place by -lr * vote."""
+    d = x.numel()
+    args = (_ptr(x, torch.float32, name="x"), _ptr(vote, torch.int8, d, "vote"), d, ctypes.c_float(lr))
+    with torch.cuda.device(x.device):
+        code = load().s3gd_apply(*args, _stream(x))
+    _check("s3gd_apply", code)
+
+
+def s3gd_step(x: torch.Tensor, grads: torch.Tensor, K: int, lr: float, ws: torch.Tensor,
+              opt_idx: Optional[torch.Tensor] = None, opt_signbits: Optional[torch.Tensor] = None,
+              opt_vote: Optional[torch.Tensor] = None) -> None:
+    """The fused step: x [d] updated in place from grads [M, d]; optional outputs as in the unfused calls."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (_ptr(x, torch.float32, d, "x"), g, M, d, K, ctypes.c_float(lr),
+            _ptr(opt_idx, torch.int32, M * K, "opt_idx"), _ptr(opt_signbits, torch.int32, M * words(K), "opt_signbits"),
+            _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(x.device):
+        code = load().s3gd_step(*args, _stream(x))
+    _check("s3gd_step", code)
+
+
+def s3gd_device_status(ws: torch.Tensor, raise_on_error: bool = True):
+    """Synchronises the current stream; returns (status code, 8 diagnostic counters)."""
+    info = (ctypes.c_uint32 * 8)()
+    w = _ptr(ws, torch.uint8, name="ws")
+    with torch.cuda.device(ws.device):
+        code = load().s3gd_device_status(w, _stream(ws), info)
+    if raise_on_error:
+        _check("s3gd_device_status", code)
+    return code, list(info)
+
+
+PHASES = ("sample", "filter", "threshold", "emit", "apply")
+
+
+def s3gd_profile_begin(max_steps: int) -> None:
+    _check("s3gd_profile_begin", load().s3gd_profile_begin(int(max_steps)))
+
+
+def s3gd_profile_end(max_steps: int):
+    """Returns (per-step list of 5 phase durations in ms, kernels enqueued since s3gd_profile_begin)."""
+    buf = (ctypes.c_float * (5 * max_steps))()
+    n = ctypes.c_int(0)
+    launches = ctypes.c_uint64(0)
+    _check("s3gd_profile_end", load().s3gd_profile_end(buf, ctypes.byref(n), ctypes.byref(launches)))
+    steps = [[buf[5 * i + k] for k in range(5)] for i in range(n.value)]
+    return steps, int(launches.value)

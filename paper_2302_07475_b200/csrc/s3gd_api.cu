@@ -1,0 +1,253 @@
+// C ABI of the library: argument checks, workspace layout, and the order in which
+// the kernels of each call are enqueued.  See include/s3gd.h for the contract.
+#include <math.h>
+
+#include "s3gd_common.cuh"
+
+namespace s3gd {
+
+// Workspace regions for (M, d, K).  The same function sizes the workspace and
+// locates the regions at run time, so the two can never disagree.
+//
+// Sampling plan (only for K <= d/4, otherwise rows are selected with full passes):
+//   n_sample entries per row are inspected; if p = K/d, the number of sampled entries
+//   that belong to the true top-K is ~ Binomial(n_sample, p) with mean s = n_sample * p.
+//   tau_lo is put at sample rank j = s + 6 sqrt(s) + 4, so the chance that fewer than K
+//   entries pass the filter is below about 1e-8; the expected number that pass is
+//   j * d / n_sample, and `cap` leaves room for 6 standard deviations, for the coarse
+//   threshold grid (2^-7 relative) and for ties.  Exceeding either bound only makes the
+//   row take the full-pass route.
+bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
+  if (M <= 0 || M > 65535 || d == 0 || d >= (1ull << 32) || K > d) return false;
+  L->M = M; L->d = d; L->K = K;
+  L->n_tiles = (uint32_t)((d + kTileElems - 1) / kTileElems);
+  L->cap = 0; L->n_sample = 0; L->j_rank = 0; L->sample_stride = 0;
+  const bool use_filter = K > 0 && K < d && K * 4 <= d;
+  if (use_filter) {
+    const double p = (double)K / (double)d;
+    double target = ceil(1024.0 / p);
+    if (target < 65536.0) target = 65536.0;
+    if (target > 1048576.0) target = 1048576.0;
+    uint64_t s_target = ((uint64_t)target + 7) / 8 * 8;
+    double j;
+    if (d <= s_target) {
+      L->n_sample = (uint32_t)d;
+      L->sample_stride = 0;
+      j = (double)K;                       // the whole row is inspected: rank K is exact
+    } else {
+      uint64_t groups = s_target / 8;
+      L->sample_stride = (uint32_t)(d / groups);
+      L->n_sample = (uint32_t)(groups * 8);
+      const double s = (double)L->n_sample * p;
+      j = ceil(s + 6.0 * sqrt(s) + 4.0);
+    }
+    if (j > (double)L->n_sample) j = (double)L->n_sample;
+    if (j < 1.0) j = 1.0;
+    L->j_rank = (uint32_t)j;
+    const double r = (double)d / (double)L->n_sample;
+    double cap = ceil(r * (j + 6.0 * sqrt(j) + 8.0) * 1.25) + 1024.0;
+    if (cap < (double)K) cap = (double)K;
+    if (cap > (double)d) cap = (double)d;
+    L->cap = (uint32_t)cap;
+  }
+  size_t off = 0;
+  L->off_hdr = off;      off = align_up(off + kHdrWords * sizeof(uint32_t), 256);
+  L->off_rows = off;     off = align_up(off + (size_t)M * sizeof(RowState), 256);
+  L->off_hist = off;     off = align_up(off + (size_t)M * kHistBins * sizeof(uint32_t), 256);
+  L->off_seg = off;      off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
+  L->off_segscan = off;  off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
+  L->off_cand = off;     off = align_up(off + (size_t)M * L->cap * sizeof(uint2), 256);
+  L->off_counter = off;  off = align_up(off + (size_t)d * sizeof(int32_t), 256);
+  L->total = off;
+  return true;
+}
+
+// ---------------------------------------------------------------- profiling
+namespace {
+struct Profiler {
+  bool on = false;
+  int max_steps = 0, n_steps = 0;
+  cudaEvent_t* ev = nullptr;          // kPhaseMarks events per recorded step
+  unsigned long long launches = 0;
+} g_prof;
+}  // namespace
+
+void prof_mark(int phase, cudaStream_t st) {
+  if (!g_prof.on || g_prof.n_steps >= g_prof.max_steps) return;
+  cudaEventRecord(g_prof.ev[(size_t)g_prof.n_steps * kPhaseMarks + phase], st);
+  if (phase == kPhaseApplied) ++g_prof.n_steps;
+}
+
+void count_launch(int n) { g_prof.launches += (unsigned long long)n; }
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+s3gd_status check_ws(const Layout& L, const void* ws, size_t ws_bytes) {
+  if (ws == nullptr || ws_bytes < L.total || !aligned(ws, 256)) return S3GD_ERR_WORKSPACE;
+  return S3GD_OK;
+}
+
+inline s3gd_status from_cuda(cudaError_t e) { return e == cudaSuccess ? S3GD_OK : S3GD_ERR_CUDA; }
+
+#define S3GD_TRY(expr)                                  \
+  do {                                                  \
+    cudaError_t e_ = (expr);                            \
+    if (e_ != cudaSuccess) return S3GD_ERR_CUDA;        \
+  } while (0)
+
+}  // namespace
+}  // namespace s3gd
+
+using namespace s3gd;
+
+extern "C" {
+
+const char* s3gd_status_string(s3gd_status st) {
+  switch (st) {
+    case S3GD_OK: return "S3GD_OK";
+    case S3GD_ERR_INVALID_ARG: return "S3GD_ERR_INVALID_ARG";
+    case S3GD_ERR_WORKSPACE: return "S3GD_ERR_WORKSPACE";
+    case S3GD_ERR_CUDA: return "S3GD_ERR_CUDA";
+    case S3GD_ERR_INDEX_RANGE: return "S3GD_ERR_INDEX_RANGE";
+    case S3GD_ERR_INTERNAL: return "S3GD_ERR_INTERNAL";
+  }
+  return "S3GD_ERR_UNKNOWN";
+}
+
+size_t s3gd_workspace_bytes(int M, uint64_t d, uint64_t K) {
+  Layout L;
+  return make_layout(M, d, K, &L) ? L.total : 0;
+}
+
+s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
+                           uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L) || grads == nullptr || !aligned(grads, 4)) return S3GD_ERR_INVALID_ARG;
+  if (K > 0 && (out_idx == nullptr || out_signbits == nullptr || !aligned(out_idx, 4) || !aligned(out_signbits, 4)))
+    return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(ws);
+  if (K == 0 || K == d) {
+    S3GD_TRY(cudaMemsetAsync(base + L.off_hdr, 0, kHdrWords * sizeof(uint32_t), st));
+    if (K == d) S3GD_TRY(launch_signplane_message(grads, M, d, out_idx, out_signbits, st));
+    return S3GD_OK;
+  }
+  S3GD_TRY(cudaMemsetAsync(out_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
+  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, st));
+}
+
+s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
+                               int8_t* out_vote, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L) || out_vote == nullptr) return S3GD_ERR_INVALID_ARG;
+  if (K > 0 && (idx == nullptr || signbits == nullptr || !aligned(idx, 4) || !aligned(signbits, 4)))
+    return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(ws);
+  uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
+  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
+  S3GD_TRY(cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st));
+  S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  S3GD_TRY(launch_vote_scatter(idx, signbits, M, K, d, counter, hdr, st));
+  S3GD_TRY(launch_counter_sign(counter, d, out_vote, st));
+  return S3GD_OK;
+}
+
+s3gd_status s3gd_apply(float* x, const int8_t* vote, uint64_t d, float lr, void* stream) {
+  if (x == nullptr || vote == nullptr || d == 0 || d >= (1ull << 32) || !aligned(x, 4)) return S3GD_ERR_INVALID_ARG;
+  return from_cuda(launch_apply(x, vote, d, lr, static_cast<cudaStream_t>(stream)));
+}
+
+s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
+                      uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L) || x == nullptr || grads == nullptr || !aligned(x, 4) || !aligned(grads, 4))
+    return S3GD_ERR_INVALID_ARG;
+  if ((opt_idx == nullptr) != (opt_signbits == nullptr)) return S3GD_ERR_INVALID_ARG;
+  if (opt_idx != nullptr && (!aligned(opt_idx, 4) || !aligned(opt_signbits, 4))) return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(ws);
+  if (K == 0 || K == d) {
+    S3GD_TRY(cudaMemsetAsync(base + L.off_hdr, 0, kHdrWords * sizeof(uint32_t), st));
+    if (K == 0) {
+      if (opt_vote) S3GD_TRY(cudaMemsetAsync(opt_vote, 0, (size_t)d, st));
+      return S3GD_OK;
+    }
+    if (opt_idx) S3GD_TRY(launch_signplane_message(grads, M, d, opt_idx, opt_signbits, st));
+    for (int ph = kPhaseStart; ph < kPhaseApplied; ++ph) prof_mark(ph, st);
+    cudaError_t e = launch_signplane_step(x, grads, M, d, lr, opt_vote, st);
+    prof_mark(kPhaseApplied, st);
+    return from_cuda(e);
+  }
+  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
+  prof_mark(kPhaseStart, st);
+  S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
+  S3GD_TRY(launch_select(grads, L, ws, opt_idx, opt_signbits, counter, st));
+  cudaError_t e = launch_counter_apply(counter, x, d, lr, opt_vote, st);
+  prof_mark(kPhaseApplied, st);
+  return from_cuda(e);
+}
+
+s3gd_status s3gd_profile_begin(int max_steps) {
+  if (max_steps <= 0 || max_steps > (1 << 20) || g_prof.on) return S3GD_ERR_INVALID_ARG;
+  const size_t n = (size_t)max_steps * kPhaseMarks;
+  g_prof.ev = new cudaEvent_t[n];
+  for (size_t i = 0; i < n; ++i) {
+    if (cudaEventCreate(&g_prof.ev[i]) != cudaSuccess) {
+      for (size_t k = 0; k < i; ++k) cudaEventDestroy(g_prof.ev[k]);
+      delete[] g_prof.ev;
+      g_prof.ev = nullptr;
+      return S3GD_ERR_CUDA;
+    }
+  }
+  g_prof.max_steps = max_steps;
+  g_prof.n_steps = 0;
+  g_prof.launches = 0;
+  g_prof.on = true;
+  return S3GD_OK;
+}
+
+s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches) {
+  if (!g_prof.on) return S3GD_ERR_INVALID_ARG;
+  s3gd_status ret = S3GD_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) ret = S3GD_ERR_CUDA;
+  for (int s = 0; s < g_prof.n_steps && ret == S3GD_OK && out_ms != nullptr; ++s) {
+    for (int ph = 0; ph + 1 < kPhaseMarks; ++ph) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, g_prof.ev[(size_t)s * kPhaseMarks + ph],
+                               g_prof.ev[(size_t)s * kPhaseMarks + ph + 1]) != cudaSuccess)
+        ret = S3GD_ERR_CUDA;
+      out_ms[(size_t)s * (kPhaseMarks - 1) + ph] = ms;
+    }
+  }
+  if (n_steps) *n_steps = g_prof.n_steps;
+  if (launches) *launches = g_prof.launches;
+  for (size_t i = 0; i < (size_t)g_prof.max_steps * kPhaseMarks; ++i) cudaEventDestroy(g_prof.ev[i]);
+  delete[] g_prof.ev;
+  g_prof = Profiler();
+  return ret;
+}
+
+s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* info) {
+  if (ws == nullptr) return S3GD_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (cudaStreamSynchronize(st) != cudaSuccess) return S3GD_ERR_CUDA;
+  if (cudaMemcpy(h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return S3GD_ERR_CUDA;
+  h[5] = h[6] = h[7] = 0;
+  if (info) for (int i = 0; i < 8; ++i) info[i] = h[i];
+  if (h[kHdrStatus] & kFlagInternal) return S3GD_ERR_INTERNAL;
+  if (h[kHdrStatus] & kFlagIndexRange) return S3GD_ERR_INDEX_RANGE;
+  return S3GD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,129 @@
+// Shared declarations of the S3GD-MV CUDA library (sm_100a): workspace layout,
+// per-row selection state, small device helpers.  Internal; the public
+// interface is include/s3gd.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "s3gd.h"
+
+namespace s3gd {
+
+// ------------------------------------------------------------------ geometry
+constexpr int kTileThreads = 256;                  // threads of a streaming CTA
+constexpr int kTileIters = 8;                      // 16-byte loads per thread per tile
+constexpr int kTileElems = kTileThreads * kTileIters * 4;   // 8192 gradient entries per tile
+constexpr int kWarpsPerTile = kTileThreads / 32;
+
+constexpr int kHistBins = 2048;                    // 11-bit digit of the first radix pass
+constexpr int kNumPasses = 3;                      // 11 + 10 + 10 bits = the 31 magnitude bits
+__host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
+__host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
+
+constexpr int kSampleBins = 32768;                 // magnitude >> 16: sign-less bf16 pattern
+constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
+
+constexpr int kSMs = 148;                          // B200
+
+// --------------------------------------------------------------- device state
+// Header at the start of the workspace (64 x uint32).
+enum HeaderWord : int {
+  kHdrStatus = 0,        // bit mask of DeviceFlag
+  kHdrExactRows = 1,     // rows that took the exact multi-pass route
+  kHdrBadIndex = 2,      // out-of-range indices skipped by the vote scatter
+  kHdrBadCount = 3,      // rows whose selection size != K
+  kHdrMaxCand = 4,       // largest candidate count of a row
+  kHdrWords = 64
+};
+enum DeviceFlag : uint32_t { kFlagIndexRange = 1u, kFlagInternal = 2u };
+
+// Selection state of one worker (row).  32 bytes.
+struct RowState {
+  uint32_t tau_lo;     // conservative magnitude threshold from the sample
+  uint32_t n_cand;     // entries with magnitude >= tau_lo found by the filter pass
+  uint32_t prefix;     // magnitude bits fixed so far by the radix passes
+  uint32_t k_rem;      // entries still to take among those matching prefix
+  uint32_t tau;        // K-th largest magnitude (valid after the last pass)
+  uint32_t take_ties;  // how many entries equal to tau are kept (lowest indices)
+  uint32_t n_emitted;  // entries written by the emit pass (checked against K)
+  uint32_t exact;      // 1: this row uses the exact multi-pass route over the whole row
+};
+
+// Byte offsets of the workspace regions; computed identically for sizing and use.
+struct Layout {
+  uint64_t d, K;
+  int M;
+  uint32_t n_tiles;      // tiles per row
+  uint32_t cap;          // candidate capacity per row
+  uint32_t n_sample;     // sampled entries per row
+  uint32_t j_rank;       // sample rank that fixes tau_lo
+  uint32_t sample_stride;  // distance between sampled groups of 8 (0: whole row sampled)
+  size_t off_hdr, off_rows, off_hist, off_seg, off_segscan, off_cand, off_counter, total;
+};
+
+bool make_layout(int M, uint64_t d, uint64_t K, Layout* L);
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ------------------------------------------------------------ device helpers
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
+__device__ __forceinline__ uint32_t lanemask_lt() {
+  uint32_t m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// Streaming loads: the gradients are read once, so keep them out of L1.
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint2 ld_stream_v2(const void* p) {
+  uint2 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+// Does this row take its top-K from the filtered candidates (true) or from the whole row?
+__device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
+  return rs.exact == 0u && rs.n_cand >= K && rs.n_cand <= cap;
+}
+#endif
+
+// ------------------------------------------------------------------ profiling
+// Optional event marks at the phase boundaries of s3gd_step (see s3gd_profile_begin).
+enum Phase : int { kPhaseStart = 0, kPhaseSampled, kPhaseFiltered, kPhaseThreshold, kPhaseEmitted, kPhaseApplied,
+                   kPhaseMarks };
+void prof_mark(int phase, cudaStream_t st);   // no-op unless profiling is on
+void count_launch(int n = 1);                 // bookkeeping of kernels enqueued by this library
+
+// ------------------------------------------------------------ kernel launchers
+// (each returns the cudaError_t of its launches; all work goes to `st`)
+cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cudaStream_t st);
+cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
+                                int32_t* counter, uint32_t* hdr, cudaStream_t st);
+cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st);
+cudaError_t launch_counter_apply(const int32_t* counter, float* x, uint64_t d, float lr, int8_t* opt_vote,
+                                 cudaStream_t st);
+cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t d, float lr, int8_t* opt_vote,
+                                  cudaStream_t st);
+cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,
+                                     uint32_t* out_signbits, cudaStream_t st);
+cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
+                                     cudaStream_t st);
+// Top-K selection of every row; writes the message if out_idx != NULL and adds the
+// votes into counter if counter != NULL.
+cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
+                          int32_t* counter, cudaStream_t st);
+
+}  // namespace s3gd

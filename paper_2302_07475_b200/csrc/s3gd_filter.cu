@@ -1,0 +1,176 @@
+// The single read of the gradients: a sampled, conservative magnitude threshold
+// per row, then one streaming pass that keeps every entry at or above it.
+//
+// Why this is exact: the true top-K of a row (Eq. (3), ties to the lower index)
+// consists of entries with magnitude >= the K-th largest magnitude.  If the
+// filter threshold tau_lo is <= that magnitude, all of them survive the filter,
+// and "survivors >= K" proves tau_lo was low enough.  The sample only decides how
+// many extra survivors there are; a bad sample costs a second route, never a wrong
+// answer (rows with too few or too many survivors take the exact multi-pass route).
+#include "s3gd_tile.cuh"
+
+namespace s3gd {
+
+namespace {
+
+__device__ __forceinline__ uint32_t mix32(uint32_t v) {   // integer finaliser, spreads group numbers
+  v ^= v >> 16; v *= 0x7FEB352Du;
+  v ^= v >> 15; v *= 0x846CA68Bu;
+  v ^= v >> 16;
+  return v;
+}
+
+// One CTA per row.  Histogram of magnitude >> 16 over n_sample entries taken in
+// groups of 8 neighbours (one 32-byte sector) spread evenly over the row, then
+// tau_lo = lower edge of the highest bin b with (#sampled >= b) >= j_rank.
+__global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                RowState* __restrict__ rows, uint32_t n_sample,
+                                                                uint32_t stride, uint32_t j_rank) {
+  extern __shared__ uint32_t s_hist[];            // kSampleBins counters
+  __shared__ uint32_t s_wsum[32];
+  __shared__ uint32_t s_pick[2];
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t row = blockIdx.x;
+  const uint32_t* rowp = gbits + (uint64_t)row * d;
+
+  for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
+  __syncthreads();
+  for (uint32_t e = tid; e < n_sample; e += 1024) {
+    uint64_t pos;
+    if (stride == 0) {
+      pos = e;
+    } else {
+      uint32_t grp = e >> 3;
+      pos = (uint64_t)grp * stride + (mix32(grp) % (stride - 7u)) + (e & 7u);
+    }
+    uint32_t key = ld_stream_u32(rowp + pos) & kAbsMask;
+    atomicAdd(&s_hist[key >> 16], 1u);
+  }
+  __syncthreads();
+
+  // warp w owns bins [1024 w, 1024 w + 1024): conflict-free strided reads
+  uint32_t part = 0;
+#pragma unroll 8
+  for (int i = 0; i < 32; ++i) part += s_hist[warp * 1024 + i * 32 + lane];
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, s);
+  if (lane == 0) s_wsum[warp] = part;
+  if (tid == 0) { s_pick[0] = 0xFFFFFFFFu; s_pick[1] = 0u; }
+  __syncthreads();
+  if (tid == 0) {
+    // highest warp range in which the count from the top reaches j_rank
+    uint32_t above = 0;
+    for (int w = 31; w >= 0; --w) {
+      if (above + s_wsum[w] >= j_rank) { s_pick[0] = (uint32_t)w; s_pick[1] = above; break; }
+      above += s_wsum[w];
+    }
+  }
+  __syncthreads();
+  const uint32_t wsel = s_pick[0];
+  if (wsel == 0xFFFFFFFFu) {                     // fewer than j_rank samples in total: keep everything
+    if (tid == 0) rows[row].tau_lo = 0u;
+    return;
+  }
+  if (warp != wsel) return;
+  // inside the chosen 1024 bins: 32 groups of 32 bins, from the top
+  uint32_t above = s_pick[1];
+  uint32_t result = 0;
+  bool found = false;
+  for (int g = 31; g >= 0 && !found; --g) {
+    uint32_t c = s_hist[wsel * 1024 + g * 32 + lane];
+    uint32_t suffix = c;                         // inclusive count of this bin and higher bins of the group
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
+      if (lane + s < 32) suffix += o;
+    }
+    uint32_t gtot = __shfl_sync(0xFFFFFFFFu, suffix, 0);
+    if (above + gtot >= j_rank) {
+      uint32_t ok = __ballot_sync(0xFFFFFFFFu, above + suffix >= j_rank);   // lanes 0..L satisfy it
+      int top = 31 - __clz(ok);                  // highest bin of the group that still reaches j_rank
+      result = wsel * 1024 + g * 32 + (uint32_t)top;
+      found = true;
+    } else {
+      above += gtot;
+    }
+  }
+  if (lane == 0) rows[row].tau_lo = result << 16;
+}
+
+// Persistent CTAs over (row, tile).  Survivors of a tile are appended to the row's
+// candidate list in ascending index order; the list position of a tile is claimed
+// with one atomic, and (position, count) is recorded per tile so that later passes
+// can walk a row's candidates in index order without sorting.
+__global__ void __launch_bounds__(kTileThreads) filter_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
+                                                              RowState* __restrict__ rows, uint2* __restrict__ cand,
+                                                              uint32_t cap, uint2* __restrict__ seg,
+                                                              uint32_t n_tiles) {
+  __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
+  __shared__ uint32_t s_base;
+  const uint64_t n_work = (uint64_t)M * n_tiles;
+  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x) {
+    const uint32_t row = (uint32_t)(w / n_tiles), t = (uint32_t)(w - (uint64_t)row * n_tiles);
+    const uint32_t* rowp = gbits + (uint64_t)row * d;
+    const uint32_t head = row_head(rowp, d);
+    const uint32_t tau_lo = rows[row].tau_lo;
+    Tile T;
+    load_tile(T, rowp, d, head, t);
+    uint32_t flags[kTileIters];
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+      uint32_t f = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) f |= (uint32_t)((T.bits[it][q] & kAbsMask) >= tau_lo) << q;
+      flags[it] = f & T.valid[it];
+    }
+    const bool head_flag = T.head_valid && (T.head_bits & kAbsMask) >= tau_lo;
+    TileRanks R;
+    tile_ranks(R, flags, head_flag, s_wtot);
+    if (threadIdx.x == 0) {
+      uint32_t base = R.tile_total ? atomicAdd(&rows[row].n_cand, R.tile_total) : 0u;
+      s_base = base;
+      seg[(uint64_t)row * n_tiles + t] = make_uint2(base, R.tile_total);
+    }
+    if (R.tile_total == 0) continue;             // uniform: every thread computed the same total
+    __syncthreads();
+    const uint32_t base = s_base;
+    uint2* out = cand + (uint64_t)row * cap;
+    if (head_flag) {
+      uint32_t pos = base + R.head_rank;
+      if (pos < cap) out[pos] = make_uint2(T.head_bits, threadIdx.x & 31);
+    }
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+      if (flags[it] == 0u) continue;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (flags[it] >> q & 1u) {
+          uint32_t pos = base + rank_of(R, flags, it, q);
+          if (pos < cap) out[pos] = make_uint2(T.bits[it][q], (uint32_t)(T.first(it) + q));
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
+                                     cudaStream_t st) {
+  // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
+  const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
+  cudaError_t e = cudaFuncSetAttribute(sample_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  sample_threshold_kernel<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  prof_mark(kPhaseSampled, st);
+  count_launch(2);
+  uint64_t n_work = (uint64_t)L.M * L.n_tiles;
+  uint64_t blocks = n_work < (uint64_t)kSMs * 8 ? n_work : (uint64_t)kSMs * 8;
+  filter_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
+  return cudaGetLastError();
+}
+
+}  // namespace s3gd

@@ -1,0 +1,367 @@
+// Second half of s3gd_select.cu: per-tile counts, their scan, the ordered emission
+// and the host-side sequencing of the whole selection.
+namespace s3gd {
+namespace {
+
+// ------------------------------------------------------------ per-tile counts
+// cnt[row][tile] = (#entries above tau, #entries equal to tau) in that tile
+// candidates: one warp per tile segment
+__global__ void __launch_bounds__(256) count_cand_kernel(const uint2* __restrict__ cand, uint32_t cap,
+                                                         const uint2* __restrict__ seg, uint32_t n_tiles,
+                                                         const RowState* __restrict__ rows, uint32_t K,
+                                                         uint2* __restrict__ cnt) {
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  if (!row_uses_candidates(rs, K, cap)) return;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t warps = gridDim.x * (blockDim.x >> 5);
+  const uint2* c = cand + (uint64_t)row * cap;
+  for (uint32_t t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
+    const uint2 sg = seg[(uint64_t)row * n_tiles + t];
+    uint32_t gt = 0, eq = 0;
+    for (uint32_t i0 = 0; i0 < sg.y; i0 += 32) {
+      uint32_t i = i0 + lane;
+      uint32_t key = (i < sg.y) ? (c[sg.x + i].x & kAbsMask) : 0u;
+      gt += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key > rs.tau));
+      eq += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key == rs.tau));
+    }
+    if (lane == 0) cnt[(uint64_t)row * n_tiles + t] = make_uint2(gt, eq);
+  }
+}
+
+// whole row: one CTA per tile
+__global__ void __launch_bounds__(kTileThreads) count_row_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                 uint32_t n_tiles, uint32_t cap,
+                                                                 const RowState* __restrict__ rows, uint32_t K,
+                                                                 uint2* __restrict__ cnt) {
+  __shared__ uint32_t s_gt[kWarpsPerTile], s_eq[kWarpsPerTile];
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  if (row_uses_candidates(rs, K, cap)) return;
+  const uint32_t* rowp = gbits + (uint64_t)row * d;
+  const uint32_t head = row_head(rowp, d);
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    Tile T;
+    load_tile(T, rowp, d, head, t);
+    uint32_t gt = 0, eq = 0;
+    if (T.head_valid) {
+      uint32_t key = T.head_bits & kAbsMask;
+      gt += key > rs.tau; eq += key == rs.tau;
+    }
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t key = T.bits[it][q] & kAbsMask;
+        uint32_t ok = T.valid[it] >> q & 1u;
+        gt += ok & (uint32_t)(key > rs.tau);
+        eq += ok & (uint32_t)(key == rs.tau);
+      }
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+      gt += __shfl_xor_sync(0xFFFFFFFFu, gt, s);
+      eq += __shfl_xor_sync(0xFFFFFFFFu, eq, s);
+    }
+    __syncthreads();
+    if (lane == 0) { s_gt[warp] = gt; s_eq[warp] = eq; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t a = 0, b = 0;
+      for (int w = 0; w < kWarpsPerTile; ++w) { a += s_gt[w]; b += s_eq[w]; }
+      cnt[(uint64_t)row * n_tiles + t] = make_uint2(a, b);
+    }
+  }
+}
+
+// ------------------------------------------------------------------- scan
+// One CTA per row.  In: cnt[tile] = (gt, eq).  Out, in place: (first output position of
+// the tile, number of entries equal to tau in earlier tiles).  A tile keeps all its
+// entries above tau, and of its entries equal to tau those whose running number
+// (in index order over the whole row) is below take_ties.
+__device__ __forceinline__ uint32_t block_exclusive_scan_1024(uint32_t v, uint32_t* s_warp, uint32_t* total) {
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) {
+    uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, s);
+    if (lane >= (uint32_t)s) inc += o;
+  }
+  __syncthreads();
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  uint32_t off = 0, tot = 0;
+  for (int w = 0; w < 32; ++w) {
+    uint32_t c = s_warp[w];
+    if ((uint32_t)w < warp) off += c;
+    tot += c;
+  }
+  *total = tot;
+  return off + inc - v;
+}
+
+__global__ void __launch_bounds__(1024) scan_kernel(uint2* __restrict__ cnt, uint32_t n_tiles,
+                                                    RowState* __restrict__ rows, uint32_t K, uint32_t cap,
+                                                    uint32_t* __restrict__ hdr) {
+  __shared__ uint32_t s_warp[32];
+  const uint32_t row = blockIdx.x, tid = threadIdx.x;
+  uint2* c = cnt + (uint64_t)row * n_tiles;
+  const uint32_t take = rows[row].take_ties;
+  const uint32_t per = (n_tiles + 1023u) / 1024u;
+  const uint32_t lo = tid * per < n_tiles ? tid * per : n_tiles;
+  const uint32_t hi = lo + per < n_tiles ? lo + per : n_tiles;
+  uint32_t eq_sum = 0;
+  for (uint32_t t = lo; t < hi; ++t) eq_sum += c[t].y;
+  uint32_t tot_eq;
+  const uint32_t eq_before = block_exclusive_scan_1024(eq_sum, s_warp, &tot_eq);
+  uint32_t sel_sum = 0, run_eq = eq_before;
+  for (uint32_t t = lo; t < hi; ++t) {
+    uint2 v = c[t];
+    uint32_t room = run_eq < take ? take - run_eq : 0u;
+    sel_sum += v.x + (v.y < room ? v.y : room);
+    run_eq += v.y;
+  }
+  uint32_t tot_sel;
+  uint32_t out = block_exclusive_scan_1024(sel_sum, s_warp, &tot_sel);
+  run_eq = eq_before;
+  for (uint32_t t = lo; t < hi; ++t) {
+    uint2 v = c[t];
+    uint32_t room = run_eq < take ? take - run_eq : 0u;
+    c[t] = make_uint2(out, run_eq);
+    out += v.x + (v.y < room ? v.y : room);
+    run_eq += v.y;
+  }
+  if (tid == 0) {
+    RowState rs = rows[row];
+    rows[row].n_emitted = tot_sel;
+    if (tot_sel != K) {
+      atomicAdd(hdr + kHdrBadCount, 1u);
+      atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
+    }
+    if (!row_uses_candidates(rs, K, cap)) atomicAdd(hdr + kHdrExactRows, 1u);
+    atomicMax(hdr + kHdrMaxCand, rs.n_cand);
+  }
+}
+
+// ------------------------------------------------------------------- emit
+struct EmitOut {
+  uint32_t* idx;        // [M x K] or NULL
+  uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
+  int32_t* counter;     // [d] or NULL
+  uint32_t K, words;
+};
+
+// candidates: one warp per tile segment, 32 entries per step.  Sign bits of the (at most
+// two) output words a step touches are gathered with a warp OR-reduction and merged
+// into the zeroed output with one atomic per word.
+__global__ void __launch_bounds__(256) emit_cand_kernel(const uint2* __restrict__ cand, uint32_t cap,
+                                                        const uint2* __restrict__ seg,
+                                                        const uint2* __restrict__ scan, uint32_t n_tiles,
+                                                        const RowState* __restrict__ rows, EmitOut o) {
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  if (!row_uses_candidates(rs, o.K, cap)) return;
+  const uint32_t lane = threadIdx.x & 31, lt = lanemask_lt();
+  const uint32_t warps = gridDim.x * (blockDim.x >> 5);
+  const uint2* c = cand + (uint64_t)row * cap;
+  for (uint32_t t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
+    const uint2 sg = seg[(uint64_t)row * n_tiles + t];
+    if (sg.y == 0) continue;
+    const uint2 sc = scan[(uint64_t)row * n_tiles + t];
+    uint32_t run_out = sc.x, run_eq = sc.y;
+    for (uint32_t i0 = 0; i0 < sg.y; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      const bool in = i < sg.y;
+      uint2 e = in ? c[sg.x + i] : make_uint2(0u, 0u);
+      const uint32_t key = e.x & kAbsMask;
+      const bool eq = in && key == rs.tau;
+      const uint32_t eqb = __ballot_sync(0xFFFFFFFFu, eq);
+      const bool sel = in && (key > rs.tau || (eq && run_eq + __popc(eqb & lt) < rs.take_ties));
+      const uint32_t selb = __ballot_sync(0xFFFFFFFFu, sel);
+      const uint32_t pos = run_out + __popc(selb & lt);
+      const uint32_t neg = e.x >> 31;
+      if (sel && pos < o.K) {
+        if (o.idx) o.idx[(uint64_t)row * o.K + pos] = e.y;
+        if (o.counter) atomicAdd(o.counter + e.y, neg ? -1 : 1);
+      }
+      if (o.signbits && selb) {
+        const uint32_t w0 = run_out >> 5;
+        const uint32_t bit = (sel && pos < o.K) ? (neg << (pos & 31)) : 0u;
+        const uint32_t v0 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 ? bit : 0u);
+        const uint32_t v1 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 + 1 ? bit : 0u);
+        if (lane == 0) {
+          if (v0) atomicOr(o.signbits + (uint64_t)row * o.words + w0, v0);
+          if (v1) atomicOr(o.signbits + (uint64_t)row * o.words + w0 + 1, v1);
+        }
+      }
+      run_out += __popc(selb);
+      run_eq += __popc(eqb);
+    }
+  }
+}
+
+// whole row: one CTA per tile; two ordered rankings (ties, then kept entries)
+__global__ void __launch_bounds__(kTileThreads) emit_row_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                uint32_t n_tiles, uint32_t cap,
+                                                                const uint2* __restrict__ scan,
+                                                                const RowState* __restrict__ rows, EmitOut o) {
+  __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  if (row_uses_candidates(rs, o.K, cap)) return;
+  const uint32_t* rowp = gbits + (uint64_t)row * d;
+  const uint32_t head = row_head(rowp, d);
+  const uint32_t lane = threadIdx.x & 31;
+  for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    const uint2 sc = scan[(uint64_t)row * n_tiles + t];
+    Tile T;
+    load_tile(T, rowp, d, head, t);
+    uint32_t eqf[kTileIters], gtf[kTileIters];
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+      uint32_t e = 0, g = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t key = T.bits[it][q] & kAbsMask;
+        e |= (uint32_t)(key == rs.tau) << q;
+        g |= (uint32_t)(key > rs.tau) << q;
+      }
+      eqf[it] = e & T.valid[it];
+      gtf[it] = g & T.valid[it];
+    }
+    const uint32_t hkey = T.head_bits & kAbsMask;
+    const bool head_eq = T.head_valid && hkey == rs.tau;
+    TileRanks Re;
+    tile_ranks(Re, eqf, head_eq, s_wtot);
+    // kept = above tau, or equal to tau with a running tie number below take_ties
+    uint32_t self[kTileIters];
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+      uint32_t s = gtf[it];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if ((eqf[it] >> q & 1u) && sc.y + rank_of(Re, eqf, it, q) < rs.take_ties) s |= 1u << q;
+      self[it] = s;
+    }
+    const bool head_sel = T.head_valid && (hkey > rs.tau || (head_eq && sc.y + Re.head_rank < rs.take_ties));
+    TileRanks Rs;
+    tile_ranks(Rs, self, head_sel, s_wtot);
+    if (Rs.tile_total == 0) continue;
+    if (head_sel) {
+      const uint32_t pos = sc.x + Rs.head_rank;
+      const uint32_t neg = T.head_bits >> 31;
+      if (pos < o.K) {
+        if (o.idx) o.idx[(uint64_t)row * o.K + pos] = lane;
+        if (o.counter) atomicAdd(o.counter + lane, neg ? -1 : 1);
+        if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
+      }
+    }
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) {
+      const uint32_t cnt_it = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(self[it]));
+      if (cnt_it == 0) continue;                  // warp-uniform
+      const uint32_t p0 = sc.x + Rs.warp_off + Rs.it_off[it];   // first output position of this warp-iteration
+      uint32_t mybits[5] = {0u, 0u, 0u, 0u, 0u};   // sign bits of my entries, by output word relative to p0 >> 5
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (self[it] >> q & 1u) {
+          const uint32_t pos = sc.x + rank_of(Rs, self, it, q);
+          if (pos < o.K) {
+            const uint32_t n = (uint32_t)(T.first(it) + q);
+            const uint32_t neg = T.bits[it][q] >> 31;
+            if (o.idx) o.idx[(uint64_t)row * o.K + pos] = n;
+            if (o.counter) atomicAdd(o.counter + n, neg ? -1 : 1);
+            const uint32_t rel = (pos >> 5) - (p0 >> 5);      // 0..4: at most 128 entries per warp-iteration
+#pragma unroll
+            for (int w = 0; w < 5; ++w)
+              if (rel == (uint32_t)w) mybits[w] |= neg << (pos & 31);
+          }
+        }
+      }
+      if (o.signbits) {
+        const uint32_t n_words = ((p0 + cnt_it - 1) >> 5) - (p0 >> 5) + 1;
+#pragma unroll
+        for (int w = 0; w < 5; ++w) {
+          if ((uint32_t)w < n_words) {
+            const uint32_t v = __reduce_or_sync(0xFFFFFFFFu, mybits[w]);
+            if (lane == 0 && v) atomicOr(o.signbits + (uint64_t)row * o.words + (p0 >> 5) + w, v);
+          }
+        }
+      }
+    }
+  }
+}
+
+inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)(v < lo ? lo : (v > hi ? hi : v)); }
+
+}  // namespace
+
+cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
+                          int32_t* counter, cudaStream_t st) {
+  char* base = static_cast<char*>(ws);
+  uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
+  RowState* rows = reinterpret_cast<RowState*>(base + L.off_rows);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(base + L.off_hist);
+  uint2* seg = reinterpret_cast<uint2*>(base + L.off_seg);
+  uint2* cnt = reinterpret_cast<uint2*>(base + L.off_segscan);
+  uint2* cand = reinterpret_cast<uint2*>(base + L.off_cand);
+  const uint32_t* gbits = reinterpret_cast<const uint32_t*>(grads);
+  const uint32_t K = (uint32_t)L.K;
+  const bool use_filter = L.cap > 0;
+  const int M = L.M;
+#define S3GD_CHECK_LAUNCH()                         \
+  do {                                              \
+    cudaError_t e_ = cudaGetLastError();            \
+    if (e_ != cudaSuccess) return e_;               \
+    count_launch();                                 \
+  } while (0)
+
+  init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K,
+                                                                                           use_filter ? 0u : 1u);
+  S3GD_CHECK_LAUNCH();
+  if (use_filter) {
+    cudaError_t e = launch_sample_and_filter(gbits, L, rows, cand, seg, st);
+    if (e != cudaSuccess) return e;
+  } else {
+    prof_mark(kPhaseSampled, st);
+  }
+  prof_mark(kPhaseFiltered, st);
+  // blocks per row for the passes over candidates / over whole rows
+  const dim3 grid_c(clampu(((uint64_t)L.cap + 4095) / 4096, 1, 64), M);
+  const dim3 grid_r(clampu(L.n_tiles, 1, ((uint64_t)kSMs * 8 + M - 1) / M), M);
+  const dim3 grid_w(clampu(((uint64_t)L.n_tiles + 7) / 8, 1, ((uint64_t)kSMs * 8 + M - 1) / M), M);
+  for (int pass = 0; pass < kNumPasses; ++pass) {
+    if (use_filter) {
+      hist_cand_kernel<<<grid_c, kHistThreads, 0, st>>>(cand, L.cap, rows, K, hist, pass);
+      S3GD_CHECK_LAUNCH();
+    }
+    hist_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, rows, K, hist, pass);
+    S3GD_CHECK_LAUNCH();
+    pick_kernel<<<M, 256, 0, st>>>(rows, hist, hdr, pass);
+    S3GD_CHECK_LAUNCH();
+  }
+  prof_mark(kPhaseThreshold, st);
+  if (use_filter) {
+    count_cand_kernel<<<grid_w, 256, 0, st>>>(cand, L.cap, seg, L.n_tiles, rows, K, cnt);
+    S3GD_CHECK_LAUNCH();
+  }
+  count_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, rows, K, cnt);
+  S3GD_CHECK_LAUNCH();
+  scan_kernel<<<M, 1024, 0, st>>>(cnt, L.n_tiles, rows, K, L.cap, hdr);
+  S3GD_CHECK_LAUNCH();
+  EmitOut o;
+  o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
+  o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
+  if (use_filter) {
+    emit_cand_kernel<<<grid_w, 256, 0, st>>>(cand, L.cap, seg, cnt, L.n_tiles, rows, o);
+    S3GD_CHECK_LAUNCH();
+  }
+  emit_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, cnt, rows, o);
+  S3GD_CHECK_LAUNCH();
+#undef S3GD_CHECK_LAUNCH
+  prof_mark(kPhaseEmitted, st);
+  return cudaSuccess;
+}
+
+}  // namespace s3gd

@@ -1,0 +1,123 @@
+// K = d: no sparsification, the step is signSGD with majority vote
+// (Section 3.3, gamma = 1).  One streaming pass over the M sign planes: every
+// thread owns a few adjacent coordinates, walks down the M rows adding
+// 1 - 2 * signbit, and updates x from the sign of the total.
+#include "s3gd_common.cuh"
+
+namespace s3gd {
+
+namespace {
+
+template <int V> struct VecLoad;
+template <> struct VecLoad<4> {
+  static __device__ __forceinline__ void load(const float* p, uint32_t (&b)[4]) {
+    uint4 v = ld_stream_v4(p);
+    b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
+  }
+};
+template <> struct VecLoad<2> {
+  static __device__ __forceinline__ void load(const float* p, uint32_t (&b)[2]) {
+    uint2 v = ld_stream_v2(p);
+    b[0] = v.x; b[1] = v.y;
+  }
+};
+template <> struct VecLoad<1> {
+  static __device__ __forceinline__ void load(const float* p, uint32_t (&b)[1]) { b[0] = ld_stream_u32(p); }
+};
+
+constexpr int kRowUnroll = 8;
+
+// V adjacent coordinates per thread; requires every row start + column to be V*4-byte aligned.
+template <int V>
+__global__ void __launch_bounds__(256) signplane_step_kernel(float* __restrict__ x, const float* __restrict__ grads,
+                                                             int M, uint64_t d, float lr,
+                                                             int8_t* __restrict__ opt_vote) {
+  const uint64_t nvec = d / V;   // host guarantees d % V == 0
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t v = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+    const float* col = grads + v * V;
+    int negs[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) negs[q] = 0;
+    int m = 0;
+    for (; m + kRowUnroll <= M; m += kRowUnroll) {
+      uint32_t b[kRowUnroll][V];
+#pragma unroll
+      for (int u = 0; u < kRowUnroll; ++u) VecLoad<V>::load(col + (uint64_t)(m + u) * d, b[u]);
+#pragma unroll
+      for (int u = 0; u < kRowUnroll; ++u)
+#pragma unroll
+        for (int q = 0; q < V; ++q) negs[q] += (int)(b[u][q] >> 31);
+    }
+    for (; m < M; ++m) {
+      uint32_t b[V];
+      VecLoad<V>::load(col + (uint64_t)m * d, b);
+#pragma unroll
+      for (int q = 0; q < V; ++q) negs[q] += (int)(b[q] >> 31);
+    }
+#pragma unroll
+    for (int q = 0; q < V; ++q) {
+      int total = M - 2 * negs[q];            // sum over workers of (+1 | -1)
+      uint64_t n = v * V + q;
+      if (opt_vote) opt_vote[n] = (int8_t)((total > 0) - (total < 0));
+      if (total > 0) x[n] = __fsub_rn(x[n], lr);
+      else if (total < 0) x[n] = __fadd_rn(x[n], lr);
+    }
+  }
+}
+
+// The transmitted form of "keep everything": idx = 0..d-1, sign bits by warp ballot.
+__global__ void __launch_bounds__(256) signplane_message_kernel(const float* __restrict__ grads, int M, uint64_t d,
+                                                                uint32_t* __restrict__ out_idx,
+                                                                uint32_t* __restrict__ out_signbits) {
+  const uint64_t words = (d + 31) / 32;
+  const uint64_t total_words = words * (uint64_t)M;
+  const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  const uint32_t lane = lane_id();
+  for (uint64_t w = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < total_words; w += warps) {
+    uint64_t m = w / words, ww = w - m * words;
+    uint64_t n = ww * 32 + lane;
+    bool neg = false;
+    if (n < d) {
+      neg = (__float_as_uint(grads[m * d + n]) >> 31) != 0u;
+      out_idx[m * d + n] = (uint32_t)n;
+    }
+    uint32_t word = __ballot_sync(0xFFFFFFFFu, neg);
+    if (lane == 0) out_signbits[w] = word;
+  }
+}
+
+inline unsigned blocks_for(uint64_t threads) {
+  uint64_t b = (threads + 255) / 256;
+  uint64_t cap = (uint64_t)kSMs * 8;
+  if (b < 1) b = 1;
+  return (unsigned)(b < cap ? b : cap);
+}
+
+}  // namespace
+
+cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t d, float lr, int8_t* opt_vote,
+                                  cudaStream_t st) {
+  uintptr_t a = reinterpret_cast<uintptr_t>(grads);
+  if (d % 4 == 0 && a % 16 == 0) {
+    signplane_step_kernel<4><<<blocks_for(d / 4), 256, 0, st>>>(x, grads, M, d, lr, opt_vote);
+    count_launch();
+  } else if (d % 2 == 0 && a % 8 == 0) {
+    signplane_step_kernel<2><<<blocks_for(d / 2), 256, 0, st>>>(x, grads, M, d, lr, opt_vote);
+    count_launch();
+  } else {
+    signplane_step_kernel<1><<<blocks_for(d), 256, 0, st>>>(x, grads, M, d, lr, opt_vote);
+    count_launch();
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,
+                                     uint32_t* out_signbits, cudaStream_t st) {
+  uint64_t warps = (uint64_t)M * ((d + 31) / 32);
+  signplane_message_kernel<<<blocks_for(warps * 32), 256, 0, st>>>(grads, M, d, out_idx, out_signbits);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace s3gd

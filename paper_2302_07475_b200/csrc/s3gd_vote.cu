@@ -1,0 +1,175 @@
+// Server side of the step: integer vote accumulation, sign, and the update of x
+// (Section 2.2 "Majority vote" and Eq. (7)).  Everything is integer work plus one
+// fp32 add per changed coordinate, so results do not depend on execution order.
+#include "s3gd_common.cuh"
+
+namespace s3gd {
+
+namespace {
+
+__device__ __forceinline__ float moved(float x, int s, float lr) {
+  // one IEEE round-to-nearest operation; __fadd_rn / __fsub_rn are never fused or reassociated
+  return s > 0 ? __fsub_rn(x, lr) : __fadd_rn(x, lr);
+}
+
+// x[n] -= lr * sgn(vote[n])
+__global__ void __launch_bounds__(256) apply_kernel(float* __restrict__ x, const int8_t* __restrict__ vote,
+                                                    uint64_t d, float lr) {
+  uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+    int s = vote[n];
+    if (s != 0) x[n] = moved(x[n], s, lr);
+  }
+}
+
+// 16 coordinates per thread step: one 16-byte load of votes, four of x.
+__global__ void __launch_bounds__(256) apply_kernel_v16(float* __restrict__ x, const int8_t* __restrict__ vote,
+                                                        uint64_t n16, float lr) {
+  uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride) {
+    uint4 v = *reinterpret_cast<const uint4*>(vote + i * 16);
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (w[q] == 0u) continue;
+      float4* px = reinterpret_cast<float4*>(x + i * 16 + q * 4);
+      float4 xv = *px;
+      int s0 = (int8_t)(w[q] & 0xFF), s1 = (int8_t)((w[q] >> 8) & 0xFF);
+      int s2 = (int8_t)((w[q] >> 16) & 0xFF), s3 = (int8_t)(w[q] >> 24);
+      if (s0) xv.x = moved(xv.x, s0, lr);
+      if (s1) xv.y = moved(xv.y, s1, lr);
+      if (s2) xv.z = moved(xv.z, s2, lr);
+      if (s3) xv.w = moved(xv.w, s3, lr);
+      *px = xv;
+    }
+  }
+}
+
+// counter[idx] += 1 - 2 * signbit for every transmitted entry
+__global__ void __launch_bounds__(256) vote_scatter_kernel(const uint32_t* __restrict__ idx,
+                                                           const uint32_t* __restrict__ signbits, int M, uint64_t K,
+                                                           uint64_t d, int32_t* __restrict__ counter,
+                                                           uint32_t* __restrict__ hdr) {
+  const uint64_t words = (K + 31) / 32;
+  const uint64_t total = (uint64_t)M * K;
+  uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  uint32_t bad = 0;
+  for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    uint64_t m = e / K, j = e - m * K;
+    uint32_t n = idx[e];
+    uint32_t neg = (signbits[m * words + (j >> 5)] >> (j & 31)) & 1u;
+    if (n < d) atomicAdd(counter + n, neg ? -1 : 1);
+    else ++bad;
+  }
+  if (bad) {
+    atomicAdd(hdr + kHdrBadIndex, bad);
+    atomicOr(hdr + kHdrStatus, (uint32_t)kFlagIndexRange);
+  }
+}
+
+__global__ void __launch_bounds__(256) counter_sign_kernel(const int32_t* __restrict__ counter, uint64_t d,
+                                                           int8_t* __restrict__ vote) {
+  uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+    int c = counter[n];
+    vote[n] = (int8_t)((c > 0) - (c < 0));
+  }
+}
+
+// sign of the counters fused with the update: 4 coordinates per thread step
+template <bool kVec>
+__global__ void __launch_bounds__(256) counter_apply_kernel(const int32_t* __restrict__ counter,
+                                                            float* __restrict__ x, uint64_t d, float lr,
+                                                            int8_t* __restrict__ opt_vote) {
+  uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  if (kVec) {
+    const uint64_t n4 = d / 4;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+      int4 c = *reinterpret_cast<const int4*>(counter + i * 4);
+      if (opt_vote) {
+        uint32_t pk = (uint32_t)(uint8_t)(int8_t)((c.x > 0) - (c.x < 0)) |
+                      ((uint32_t)(uint8_t)(int8_t)((c.y > 0) - (c.y < 0)) << 8) |
+                      ((uint32_t)(uint8_t)(int8_t)((c.z > 0) - (c.z < 0)) << 16) |
+                      ((uint32_t)(uint8_t)(int8_t)((c.w > 0) - (c.w < 0)) << 24);
+        *reinterpret_cast<uint32_t*>(opt_vote + i * 4) = pk;
+      }
+      if ((c.x | c.y | c.z | c.w) == 0) continue;
+      float4* px = reinterpret_cast<float4*>(x + i * 4);
+      float4 xv = *px;
+      if (c.x) xv.x = moved(xv.x, c.x, lr);
+      if (c.y) xv.y = moved(xv.y, c.y, lr);
+      if (c.z) xv.z = moved(xv.z, c.z, lr);
+      if (c.w) xv.w = moved(xv.w, c.w, lr);
+      *px = xv;
+    }
+    // ragged tail (d % 4 entries)
+    uint64_t n = n4 * 4 + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (n < d) {
+      int c = counter[n];
+      if (opt_vote) opt_vote[n] = (int8_t)((c > 0) - (c < 0));
+      if (c) x[n] = moved(x[n], c, lr);
+    }
+  } else {
+    for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+      int c = counter[n];
+      if (opt_vote) opt_vote[n] = (int8_t)((c > 0) - (c < 0));
+      if (c) x[n] = moved(x[n], c, lr);
+    }
+  }
+}
+
+inline unsigned grid_for(uint64_t items, int per_block, int max_blocks) {
+  uint64_t b = (items + per_block - 1) / per_block;
+  if (b < 1) b = 1;
+  if (b > (uint64_t)max_blocks) b = max_blocks;
+  return (unsigned)b;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cudaStream_t st) {
+  if (aligned(x, 16) && aligned(vote, 16) && d >= 16) {
+    uint64_t n16 = d / 16;
+    apply_kernel_v16<<<grid_for(n16, 256, kSMs * 8), 256, 0, st>>>(x, vote, n16, lr);
+    count_launch();
+    uint64_t done = n16 * 16;
+    if (done < d) apply_kernel<<<1, 256, 0, st>>>(x + done, vote + done, d - done, lr);
+    if (done < d) count_launch();
+  } else {
+    apply_kernel<<<grid_for(d, 256, kSMs * 8), 256, 0, st>>>(x, vote, d, lr);
+    count_launch();
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
+                                int32_t* counter, uint32_t* hdr, cudaStream_t st) {
+  uint64_t total = (uint64_t)M * K;
+  if (total == 0) return cudaSuccess;
+  vote_scatter_kernel<<<grid_for(total, 256, kSMs * 16), 256, 0, st>>>(idx, signbits, M, K, d, counter, hdr);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st) {
+  counter_sign_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, d, vote);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_counter_apply(const int32_t* counter, float* x, uint64_t d, float lr, int8_t* opt_vote,
+                                 cudaStream_t st) {
+  bool vec = aligned(x, 16) && aligned(counter, 16) && (opt_vote == nullptr || aligned(opt_vote, 4)) && d >= 4;
+  if (vec) {
+    counter_apply_kernel<true><<<grid_for(d / 4, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
+    count_launch();
+  } else {
+    counter_apply_kernel<false><<<grid_for(d, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
+    count_launch();
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace s3gd

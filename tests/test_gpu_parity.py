@@ -1,0 +1,301 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, bit for bit.
+
+Indices, sign bits, votes and the updated x are all integers or a single fp32
+rounding, so the bar is exact equality (tolerance 0) on every output.
+Small and medium cases are compared element by element with the definitional
+oracle; the full-size workloads are compared with the oracle's threshold route
+(itself pinned to the definition on CPU) on every row, with the definition on
+sampled rows, and with the O(d) certificate check.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2302_07475_b200 as S
+from oracle import s3gd_oracle as O
+from paper_2302_07475_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def u32(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32)
+
+
+def bits(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+class Runner:
+    """Buffers for one (M, d, K) and the two ways through the library."""
+
+    def __init__(self, M, d, K):
+        self.M, self.d, self.K = M, d, K
+        self.ws = S.alloc_workspace(M, d, K, DEV)
+        self.ws.fill_(0xA5)                       # the library must not rely on a clean workspace
+        self.idx = torch.full((M, max(K, 1)), -1, dtype=torch.int32, device=DEV)[:, :K].contiguous()
+        self.sgn = torch.full((M, max(S.binding.words(K), 1)), -1, dtype=torch.int32, device=DEV)[:, :S.binding.words(K)].contiguous()
+        self.vote = torch.full((d,), 77, dtype=torch.int8, device=DEV)
+
+    def unfused(self, grads, x, lr):
+        x = x.clone()
+        S.s3gd_topk_sign(grads, self.K, self.idx, self.sgn, self.ws)
+        code, info = S.s3gd_device_status(self.ws)
+        S.s3gd_majority_vote(self.idx, self.sgn, self.M, self.K, self.d, self.vote, self.ws)
+        S.s3gd_apply(x, self.vote, lr)
+        S.s3gd_device_status(self.ws)
+        return u32(self.idx), u32(self.sgn), self.vote.cpu().numpy().copy(), x.cpu().numpy(), info
+
+    def fused(self, grads, x, lr, outputs=True):
+        x = x.clone()
+        if outputs:
+            self.idx.fill_(-1); self.sgn.fill_(-1); self.vote.fill_(77)
+            S.s3gd_step(x, grads, self.K, lr, self.ws, self.idx, self.sgn, self.vote)
+        else:
+            S.s3gd_step(x, grads, self.K, lr, self.ws)
+        code, info = S.s3gd_device_status(self.ws)
+        if outputs:
+            return u32(self.idx), u32(self.sgn), self.vote.cpu().numpy().copy(), x.cpu().numpy(), info
+        return None, None, None, x.cpu().numpy(), info
+
+
+def check_all(grads_t, x_t, K, lr, oracle_topk=O.topk_sign, tag=""):
+    M, d = grads_t.shape
+    g = grads_t.cpu().numpy()
+    x = x_t.cpu().numpy()
+    idx_o, sgn_o = oracle_topk(g, K)
+    vote_o, bad = O.majority_vote(idx_o, sgn_o, M, K, d)
+    assert bad == 0
+    x_o = O.apply_vote(x, vote_o, lr)
+    r = Runner(M, d, K)
+    for name, out in (("unfused", r.unfused(grads_t, x_t, lr)), ("fused+outputs", r.fused(grads_t, x_t, lr, True)),
+                      ("fused", r.fused(grads_t, x_t, lr, False))):
+        idx, sgn, vote, xn, info = out
+        if idx is not None:
+            assert np.array_equal(idx, idx_o), f"{tag} {name}: indices differ"
+            assert np.array_equal(sgn, sgn_o), f"{tag} {name}: sign bits differ"
+            assert np.array_equal(vote, vote_o), f"{tag} {name}: votes differ"
+        assert np.array_equal(bits(xn), bits(x_o)), f"{tag} {name}: updated x differs"
+    return info
+
+
+# ------------------------------------------------------------------ workloads
+def test_tiny_workload():
+    s = W.SPECS["tiny"]
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    info = check_all(g, x, s.Ks[0], s.lr, tag="tiny")
+    assert info[1] == 0            # every row served by the filtered candidates
+
+
+@pytest.mark.parametrize("K", W.SPECS["small_cnn"].Ks)
+def test_small_cnn_ten_steps(K):
+    s = W.SPECS["small_cnn"]
+    x_gpu = W.make_x(s, DEV)
+    x_cpu = x_gpu.cpu().numpy()
+    ws = S.alloc_workspace(s.M, s.d, K, DEV)
+    for step in range(s.steps):
+        g = W.make_grads(s, DEV, step=step)
+        S.s3gd_step(x_gpu, g, K, s.lr, ws)
+        S.s3gd_device_status(ws)
+        x_cpu, _, _, _ = O.step(x_cpu, g.cpu().numpy(), K, s.lr)
+        assert np.array_equal(bits(x_gpu.cpu().numpy()), bits(x_cpu)), f"step {step}"
+    # and once through the unfused calls on the last step's gradients
+    check_all(g, W.make_x(s, DEV), K, s.lr, oracle_topk=O.topk_sign_threshold, tag="small_cnn")
+
+
+@pytest.mark.parametrize("name,d,M,Ks", [
+    ("resnet18", 300_007, 7, (300, 3_001, 75_001, 75_002, 300_007)),
+    ("resnet50_ties", 262_144 + 6, 5, (26, 262, 2_621, 26_215)),
+    ("large", 1_000_003, 3, (1_000, 250_000)),
+])
+def test_reduced_workloads_against_definition(name, d, M, Ks):
+    s = W.spec(name, d=d, M=M)
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    for K in Ks:
+        check_all(g, x, K, s.lr, tag=f"{name} K={K}")
+
+
+def _full_size(name, Ks, sample_rows):
+    s = W.SPECS[name]
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    g_cpu = g.cpu().numpy()
+    for K in Ks:
+        if K == s.d:
+            idx_o = sgn_o = None
+            neg = (g_cpu.view(np.uint32) >> 31).astype(np.int64).sum(axis=0)
+            total = s.M - 2 * neg                         # Section 3.3, gamma = 1: plain sign counting
+            vote_o = (total > 0).astype(np.int8) - (total < 0).astype(np.int8)
+        else:
+            idx_o, sgn_o = O.topk_sign_threshold(g_cpu, K)
+            for m in sample_rows:                          # the definition itself on a few rows
+                i_d, s_d = O.topk_sign(g_cpu[m:m + 1], K)
+                assert np.array_equal(i_d[0], idx_o[m]) and np.array_equal(s_d[0], sgn_o[m])
+            vote_o, _ = O.majority_vote(idx_o, sgn_o, s.M, K, s.d)
+        x_o = O.apply_vote(x.cpu().numpy(), vote_o, s.lr)
+        ws = S.alloc_workspace(s.M, s.d, K, DEV)
+        xg = x.clone()
+        vote = torch.empty(s.d, dtype=torch.int8, device=DEV)
+        if K == s.d:
+            S.s3gd_step(xg, g, K, s.lr, ws, None, None, vote)
+        else:
+            idx = torch.empty((s.M, K), dtype=torch.int32, device=DEV)
+            sgn = torch.empty((s.M, S.binding.words(K)), dtype=torch.int32, device=DEV)
+            S.s3gd_step(xg, g, K, s.lr, ws, idx, sgn, vote)
+        code, info = S.s3gd_device_status(ws)
+        assert np.array_equal(vote.cpu().numpy(), vote_o), f"{name} K={K}: votes differ"
+        assert np.array_equal(bits(xg.cpu().numpy()), bits(x_o)), f"{name} K={K}: x differs"
+        if K != s.d:
+            idx_g, sgn_g = u32(idx), u32(sgn)
+            assert np.array_equal(idx_g, idx_o), f"{name} K={K}: indices differ"
+            assert np.array_equal(sgn_g, sgn_o), f"{name} K={K}: sign bits differ"
+            for m in sample_rows:
+                assert O.check_topk_sign_row(g_cpu[m], K, idx_g[m], sgn_g[m]) == ""
+            # the launch configuration the benchmark times: no optional outputs
+            xb = x.clone()
+            S.s3gd_step(xb, g, K, s.lr, ws)
+            S.s3gd_device_status(ws)
+            assert np.array_equal(bits(xb.cpu().numpy()), bits(x_o)), f"{name} K={K}: x differs (no outputs)"
+            if K * 100 <= s.d:
+                assert info[1] == 0, f"{name} K={K}: {info[1]} rows left the single-read route"
+        del ws
+
+
+def test_resnet18_full_size():
+    _full_size("resnet18", W.SPECS["resnet18"].Ks, sample_rows=(0, 57))
+
+
+def test_resnet50_tie_stress_full_size():
+    _full_size("resnet50_ties", W.SPECS["resnet50_ties"].Ks, sample_rows=(31,))
+
+
+@pytest.mark.skipif(os.environ.get("S3GD_TEST_LARGE") != "1", reason="67 GB case: set S3GD_TEST_LARGE=1")
+def test_large_full_size_row_by_row():
+    """d = 2.1e9, M = 8: the rows are generated, stepped and then certified one by one on the host."""
+    s = W.SPECS["large"]
+    K = s.Ks[0]
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    x0 = x.cpu().numpy().copy()
+    ws = S.alloc_workspace(s.M, s.d, K, DEV)
+    idx = torch.empty((s.M, K), dtype=torch.int32, device=DEV)
+    sgn = torch.empty((s.M, S.binding.words(K)), dtype=torch.int32, device=DEV)
+    S.s3gd_step(x, g, K, s.lr, ws, idx, sgn, None)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0
+    idx_g, sgn_g = u32(idx), u32(sgn)
+    idx_o = np.zeros_like(idx_g); sgn_o = np.zeros_like(sgn_g)
+    for m in range(s.M):
+        row = g[m].cpu().numpy()
+        i_o, s_o = O.topk_sign_threshold(row[None, :], K)
+        idx_o[m], sgn_o[m] = i_o[0], s_o[0]
+        assert np.array_equal(idx_g[m], idx_o[m]) and np.array_equal(sgn_g[m], sgn_o[m]), f"row {m}"
+        del row
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, s.M, K, s.d)
+    x_o = O.apply_vote(x0, vote_o, s.lr)
+    assert np.array_equal(bits(x.cpu().numpy()), bits(x_o))
+
+
+def test_large_recipe_reduced_64bit_offsets():
+    """Same recipe, M*d just above 2^32 bytes of offsets: row offsets must be 64-bit."""
+    s = W.spec("large", d=268_435_459, M=5)             # M*d*4 bytes = 5.4 GB, m*d exceeds 2^30 elements
+    K = 268_435
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    g_last = g[s.M - 1].cpu().numpy()
+    ws = S.alloc_workspace(s.M, s.d, K, DEV)
+    idx = torch.empty((s.M, K), dtype=torch.int32, device=DEV)
+    sgn = torch.empty((s.M, S.binding.words(K)), dtype=torch.int32, device=DEV)
+    S.s3gd_topk_sign(g, K, idx, sgn, ws)
+    S.s3gd_device_status(ws)
+    i_o, s_o = O.topk_sign_threshold(g_last[None, :], K)
+    assert np.array_equal(u32(idx)[s.M - 1], i_o[0]) and np.array_equal(u32(sgn)[s.M - 1], s_o[0])
+    assert O.check_topk_sign_row(g_last, K, u32(idx)[s.M - 1], u32(sgn)[s.M - 1]) == ""
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("kind", ["all_equal", "zeros", "few_levels", "one_hot", "special", "ramp", "ramp_down"])
+def test_degenerate_inputs(kind):
+    for (M, d) in ((1, 1), (2, 5), (3, 31), (3, 33), (4, 1537), (2, 8192), (3, 8193), (2, 40_001)):
+        g = W.edge_case_grads(kind, M, d, DEV)
+        x = torch.linspace(-1, 1, d, device=DEV)
+        for K in sorted({0, 1, min(d, 7), d // 4, d // 4 + 1, d // 2, d - 1, d}):
+            if K < 0:
+                continue
+            check_all(g, x, K, 0.01, tag=f"{kind} M={M} d={d} K={K}")
+
+
+def test_rows_not_16_byte_aligned():
+    """d = 1537 and a base pointer offset by 1..3 floats: every row starts at a different alignment."""
+    M, d = 5, 1537 * 7
+    for off in (0, 1, 2, 3):
+        big = torch.randn(M * d + 8, device=DEV, generator=torch.Generator(DEV).manual_seed(off))
+        g = big[off:off + M * d].view(M, d)
+        assert g.is_contiguous() and g.data_ptr() % 16 == (big.data_ptr() + 4 * off) % 16
+        x = torch.zeros(d, device=DEV)
+        for K in (11, 1000, d // 2, d):
+            check_all(g, x, K, 0.5, tag=f"offset {off} K={K}")
+
+
+def test_rows_that_leave_the_single_read_route():
+    """All magnitudes equal: the filter keeps everything, overflows its buffer, and the row is redone exactly."""
+    M, d, K = 3, 100_000, 1000
+    g = W.edge_case_grads("all_equal", M, d, DEV)
+    info = check_all(g, torch.zeros(d, device=DEV), K, 0.1, tag="overflow")
+    assert info[1] == M
+    # mixed: one ordinary row between two constant rows
+    g[1] = torch.randn(d, device=DEV)
+    info = check_all(g, torch.zeros(d, device=DEV), K, 0.1, tag="mixed")
+    assert info[1] == M - 1
+
+
+def test_majority_vote_semantics_and_range_flag():
+    d, M, K = 10, 2, 4
+    idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)
+    sgn = torch.tensor([[0b0110], [0b0001]], dtype=torch.int32, device=DEV)
+    vote = torch.empty(d, dtype=torch.int8, device=DEV)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    S.s3gd_majority_vote(idx, sgn, M, K, d, vote, ws)
+    code, info = S.s3gd_device_status(ws, raise_on_error=False)
+    want, bad = O.majority_vote(u32(idx), u32(sgn), M, K, d)
+    assert vote.cpu().numpy().tolist() == want.tolist()
+    assert code == 4 and info[2] == bad == 1                # S3GD_ERR_INDEX_RANGE, one index skipped
+    # a later clean call clears the record
+    idx[1, 3] = 0
+    S.s3gd_majority_vote(idx, sgn, M, K, d, vote, ws)
+    code, info = S.s3gd_device_status(ws)
+    assert code == 0 and info[2] == 0
+
+
+def test_apply_leaves_unvoted_bits_alone():
+    xb = np.array([0x7FC12345, 0x80000000, 0x00000001, 0x3F800000, 0x7F800000, 0x3DCCCCCD] * 7, dtype=np.uint32)
+    d = xb.shape[0]
+    x = torch.from_numpy(xb.view(np.float32).copy()).to(DEV)
+    for pattern in (np.zeros(d, np.int8), np.ones(d, np.int8), -np.ones(d, np.int8),
+                    np.resize(np.array([0, 1, -1, 5, -7], np.int8), d)):
+        xx = x.clone()
+        S.s3gd_apply(xx, torch.from_numpy(pattern).to(DEV), 0.3)
+        torch.cuda.synchronize()
+        want = O.apply_vote(xb.view(np.float32), np.sign(pattern).astype(np.int8), 0.3)
+        got = xx.cpu().numpy()
+        same = bits(got) == bits(want)
+        nan_both = np.isnan(got) & np.isnan(want)
+        assert np.all(same | nan_both)
+        assert np.array_equal(bits(got)[pattern == 0], xb[pattern == 0])
+
+
+def test_repeatable():
+    s = W.spec("resnet18", d=500_000, M=9)
+    g = W.make_grads(s, DEV)
+    x = W.make_x(s, DEV)
+    r = Runner(s.M, s.d, 5000)
+    a = r.fused(g, x, 1e-3, True)
+    for _ in range(3):
+        b = r.fused(g, x, 1e-3, True)
+        for u, v in zip(a[:4], b[:4]):
+            assert np.array_equal(bits(u) if u.dtype == np.float32 else u, bits(v) if v.dtype == np.float32 else v)
