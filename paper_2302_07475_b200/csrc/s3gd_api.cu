@@ -10,7 +10,7 @@ namespace s3gd {
 // locates the regions at run time, so the two can never disagree.
 //
 // Sampling plan (only for K <= d/4, otherwise rows are selected with full passes):
-//   n_sample entries per row are inspected; if p = K/d, the number of sampled entries
+//   n_sample = 65536 entries per row are inspected (all of them for short rows); if p = K/d, the number of sampled entries
 //   that belong to the true top-K is ~ Binomial(n_sample, p) with mean s = n_sample * p.
 //   tau_lo is put at sample rank j = s + 6 sqrt(s) + 4, so the chance that fewer than K
 //   entries pass the filter is below about 1e-8; the expected number that pass is
@@ -25,19 +25,16 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   const bool use_filter = K > 0 && K < d && K * 4 <= d;
   if (use_filter) {
     const double p = (double)K / (double)d;
-    double target = ceil(1024.0 / p);
-    if (target < 65536.0) target = 65536.0;
-    if (target > 1048576.0) target = 1048576.0;
-    uint64_t s_target = ((uint64_t)target + 7) / 8 * 8;
+    const uint64_t s_target = 65536;       // 2048 chunks of 32 neighbouring entries
     double j;
-    if (d <= s_target) {
+    if (d <= 2 * s_target) {
       L->n_sample = (uint32_t)d;
       L->sample_stride = 0;
       j = (double)K;                       // the whole row is inspected: rank K is exact
     } else {
-      uint64_t groups = s_target / 8;
-      L->sample_stride = (uint32_t)(d / groups);
-      L->n_sample = (uint32_t)(groups * 8);
+      const uint64_t chunks = s_target / 32;
+      L->sample_stride = (uint32_t)(d / chunks);
+      L->n_sample = (uint32_t)(chunks * 32);
       const double s = (double)L->n_sample * p;
       j = ceil(s + 6.0 * sqrt(s) + 4.0);
     }

@@ -20,9 +20,13 @@ __device__ __forceinline__ uint32_t mix32(uint32_t v) {   // integer finaliser, 
   return v;
 }
 
-// One CTA per row.  Histogram of magnitude >> 16 over n_sample entries taken in
-// groups of 8 neighbours (one 32-byte sector) spread evenly over the row, then
+// One CTA per row.  Histogram of magnitude >> 16 over n_sample entries taken as
+// chunks of 32 neighbours (one 128-byte line, so the sample costs its own bytes and
+// no more) spread evenly over the row with a hashed offset inside each stride, then
 // tau_lo = lower edge of the highest bin b with (#sampled >= b) >= j_rank.
+constexpr int kChunk = 32;
+constexpr int kSampleUnroll = 8;
+
 __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 RowState* __restrict__ rows, uint32_t n_sample,
                                                                 uint32_t stride, uint32_t j_rank) {
@@ -35,16 +39,24 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
 
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
   __syncthreads();
-  for (uint32_t e = tid; e < n_sample; e += 1024) {
-    uint64_t pos;
-    if (stride == 0) {
-      pos = e;
-    } else {
-      uint32_t grp = e >> 3;
-      pos = (uint64_t)grp * stride + (mix32(grp) % (stride - 7u)) + (e & 7u);
+  if (stride == 0) {                              // short row: every entry is inspected
+    for (uint32_t e = tid; e < n_sample; e += 1024) atomicAdd(&s_hist[(rowp[e] & kAbsMask) >> 16], 1u);
+  } else {
+    const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
+    for (uint32_t c0 = warp; c0 < n_chunks; c0 += 32 * kSampleUnroll) {
+      uint32_t v[kSampleUnroll];
+#pragma unroll
+      for (int u = 0; u < kSampleUnroll; ++u) {
+        const uint32_t c = c0 + 32 * u;
+        if (c < n_chunks) {
+          const uint64_t pos = (uint64_t)c * stride + (mix32(c) % (stride - (kChunk - 1))) + lane;
+          v[u] = __ldg(rowp + pos);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kSampleUnroll; ++u)
+        if (c0 + 32 * u < n_chunks) atomicAdd(&s_hist[(v[u] & kAbsMask) >> 16], 1u);
     }
-    uint32_t key = ld_stream_u32(rowp + pos) & kAbsMask;
-    atomicAdd(&s_hist[key >> 16], 1u);
   }
   __syncthreads();
 
