@@ -182,6 +182,21 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------- multi-rank plumbing
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a short list of floats over all ranks (identity without a process group)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(world, M, d, steps, ms_total):
+    """Elements/s of the whole job: every rank steps its own M x d replica; time is the slowest rank's."""
+    return world * M * d * steps / (ms_total * 1e-3)
+
+
 # --------------------------------------------------------------------------- GPU side
 def run_ours(args):
     import torch
@@ -262,15 +277,12 @@ def run_ours(args):
         e2e_ms = None
         e2e_err = str(exc).splitlines()[0]
 
-    times = torch.tensor([ms_total, e2e_ms if e2e_ms is not None else 0.0], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_max = float(times[0]), float(times[1])
+    ms_total, e2e_max = max_over_ranks([ms_total, e2e_ms if e2e_ms is not None else 0.0], dist, dev)
 
     if rank == 0:
         elems_per_step = world * M * d
         ms_step = ms_total / args.steps
-        value = elems_per_step / (ms_step * 1e-3)
+        value = whole_job_value(world, M, d, args.steps, ms_total)
         b_grad, b_dense, b_min = byte_models(M, d, K)
         peak, peak_kind = measured_peak()
         mean_phase = [sum(p[k] for p in phases) / max(len(phases), 1) for k in range(5)]
