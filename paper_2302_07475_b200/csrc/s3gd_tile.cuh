@@ -3,9 +3,10 @@
 //
 // A row of d fp32 values starts at an address that is only 4-byte aligned in
 // general (d need not be a multiple of 4).  `head` = number of leading entries
-// before the first 16-byte boundary (0..3).  Tile t covers the entries
-// [head + t*kTileElems, head + (t+1)*kTileElems) with 16-byte loads; tile 0 also
-// owns the `head` leading entries, which lanes 0..2 of warp 0 load as scalars.
+// before the first 128-byte boundary (0..31).  Tile t covers the entries
+// [head + t*kTileElems, head + (t+1)*kTileElems) with 16-byte loads, so every tile
+// starts on a cache line; tile 0 also owns the `head` leading entries, which the
+// low lanes of warp 0 load as scalars.
 //
 // Inside a tile warp w owns the contiguous 1024 entries starting at w*1024, and in
 // iteration `it` lane l holds entries w*1024 + it*128 + l*4 + {0,1,2,3}.  So the
@@ -28,7 +29,7 @@ struct Tile {
 };
 
 __device__ __forceinline__ uint32_t row_head(const uint32_t* rowp, uint64_t d) {
-  uint32_t h = (uint32_t)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(rowp) & 15u)) & 15u) >> 2);
+  uint32_t h = (uint32_t)(((128u - (uint32_t)(reinterpret_cast<uintptr_t>(rowp) & 127u)) & 127u) >> 2);
   return (uint64_t)h < d ? h : (uint32_t)d;
 }
 
