@@ -51,7 +51,8 @@ typedef enum s3gd_status {
   S3GD_ERR_WORKSPACE = 2,   /* workspace NULL, smaller than s3gd_workspace_bytes(), or not 256-byte aligned */
   S3GD_ERR_CUDA = 3,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
   S3GD_ERR_INDEX_RANGE = 4, /* device: an index >= d was given to s3gd_majority_vote (skipped) */
-  S3GD_ERR_INTERNAL = 5     /* device: a selection did not produce exactly K entries */
+  S3GD_ERR_INTERNAL = 5,    /* device: a selection did not produce exactly K entries */
+  S3GD_ERR_TOO_LARGE = 6    /* s3gd_majority_vote_noalloc: d exceeds s3gd_noalloc_max_d() */
 } s3gd_status;
 
 /* Human-readable name of a status code.  Host.  Never NULL. */
@@ -132,6 +133,33 @@ S3GD_API s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, 
  *   [4] largest candidate count of a row  [5..7] reserved (0)
  */
 S3GD_API s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* info);
+
+/*
+ * Majority vote without any caller-provided scratch (the paper has no counterpart: this is
+ * a convenience of this library, same result as s3gd_majority_vote).
+ *
+ * For callers that cannot allocate device memory where they vote -- code running inside
+ * another framework's callback that must not call into its allocator, a plug-in that is
+ * handed nothing but input and output buffers, a process whose device memory is already
+ * fully owned by a pool it does not control.  The d int32 counters live in a fixed array
+ * inside this library (16 MiB + 256 bytes on every GPU that loads it, held until the
+ * process exits), so d is limited: s3gd_noalloc_max_d() = 4,194,304 coordinates; a larger
+ * d returns S3GD_ERR_TOO_LARGE and nothing is enqueued.  The call allocates and frees
+ * nothing.
+ *
+ *  idx, signbits, M, K, d, out_vote   as for s3gd_majority_vote (dev pointers)
+ *  opt_bad_count  dev or NULL  receives the number of indices >= d that were skipped
+ *
+ * The first call on each device looks up the device address of the built-in array (a
+ * runtime query, no allocation) with that device current; make that first call outside
+ * any stream capture.  All calls on a device share the one array: it is cleared at the
+ * start of every call, so results never depend on earlier calls, but two calls that may
+ * run on the GPU at the same time (different streams) race on it -- serialise them.
+ */
+S3GD_API uint64_t s3gd_noalloc_max_d(void);
+S3GD_API s3gd_status s3gd_majority_vote_noalloc(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K,
+                                                uint64_t d, int8_t* out_vote, uint32_t* opt_bad_count,
+                                                void* stream);
 
 /*
  * Measurement aid (the paper reports no timings; this has no counterpart there).

@@ -19,11 +19,12 @@ LIB_PATH = os.path.join(_PKG, "libs3gd.so")
 S3GD_OK = 0
 STATUS_NAMES = {
     0: "S3GD_OK", 1: "S3GD_ERR_INVALID_ARG", 2: "S3GD_ERR_WORKSPACE", 3: "S3GD_ERR_CUDA",
-    4: "S3GD_ERR_INDEX_RANGE", 5: "S3GD_ERR_INTERNAL",
+    4: "S3GD_ERR_INDEX_RANGE", 5: "S3GD_ERR_INTERNAL", 6: "S3GD_ERR_TOO_LARGE",
 }
 
 EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
-           "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end")
+           "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
+           "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc")
 
 
 class S3gdError(RuntimeError):
@@ -65,6 +66,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_profile_begin.argtypes = [ctypes.c_int]
     lib.s3gd_profile_end.restype = ctypes.c_int
     lib.s3gd_profile_end.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    lib.s3gd_noalloc_max_d.restype = ctypes.c_uint64
+    lib.s3gd_noalloc_max_d.argtypes = []
+    lib.s3gd_majority_vote_noalloc.restype = ctypes.c_int
+    lib.s3gd_majority_vote_noalloc.argtypes = [u32p, u32p, ctypes.c_int, u64, u64, vp, vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -181,3 +186,21 @@ def s3gd_profile_end(max_steps: int):
     _check("s3gd_profile_end", load().s3gd_profile_end(buf, ctypes.byref(n), ctypes.byref(launches)))
     steps = [[buf[5 * i + k] for k in range(5)] for i in range(n.value)]
     return steps, int(launches.value)
+
+
+def s3gd_noalloc_max_d() -> int:
+    return int(load().s3gd_noalloc_max_d())
+
+
+def s3gd_majority_vote_noalloc(idx: torch.Tensor, signbits: torch.Tensor, M: int, K: int, d: int,
+                               out_vote: torch.Tensor, opt_bad_count: Optional[torch.Tensor] = None) -> None:
+    """Majority vote whose counters live inside the library: no workspace argument, nothing allocated.
+
+    For callers that cannot obtain device memory where they vote (see include/s3gd.h).  d must not
+    exceed s3gd_noalloc_max_d(); calls on one device share the built-in counters, so do not overlap them.
+    """
+    args = (_ptr(idx, torch.int32, M * K, "idx"), _ptr(signbits, torch.int32, M * words(K), "signbits"), M, K, d,
+            _ptr(out_vote, torch.int8, d, "out_vote"), _ptr(opt_bad_count, torch.int32, 1, "opt_bad_count"))
+    with torch.cuda.device(out_vote.device):
+        code = load().s3gd_majority_vote_noalloc(*args, _stream(out_vote))
+    _check("s3gd_majority_vote_noalloc", code)

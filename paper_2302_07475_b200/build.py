@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libs3gd.so")
-SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu"]
+SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu", "s3gd_noalloc.cu"]
 HEADERS = ["s3gd_common.cuh", "s3gd_tile.cuh", "s3gd_select_emit.inl"]
 
 
@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [
         _nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
         "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-shared",
-        "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+        "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-DS3GD_NOALLOC_MAX_D=4194304ull",
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]

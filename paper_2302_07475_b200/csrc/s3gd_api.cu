@@ -109,6 +109,7 @@ const char* s3gd_status_string(s3gd_status st) {
     case S3GD_ERR_CUDA: return "S3GD_ERR_CUDA";
     case S3GD_ERR_INDEX_RANGE: return "S3GD_ERR_INDEX_RANGE";
     case S3GD_ERR_INTERNAL: return "S3GD_ERR_INTERNAL";
+    case S3GD_ERR_TOO_LARGE: return "S3GD_ERR_TOO_LARGE";
   }
   return "S3GD_ERR_UNKNOWN";
 }
