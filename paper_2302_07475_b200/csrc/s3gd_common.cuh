@@ -39,7 +39,7 @@ enum HeaderWord : int {
 };
 enum DeviceFlag : uint32_t { kFlagIndexRange = 1u, kFlagInternal = 2u };
 
-// Selection state of one worker (row).  32 bytes.
+// Selection state of one worker (row).  64 bytes.
 struct RowState {
   uint32_t tau_lo;     // conservative magnitude threshold from the sample
   uint32_t n_cand;     // entries with magnitude >= tau_lo found by the filter pass
@@ -49,6 +49,9 @@ struct RowState {
   uint32_t take_ties;  // how many entries equal to tau are kept (lowest indices)
   uint32_t n_emitted;  // entries written by the emit pass (checked against K)
   uint32_t exact;      // 1: this row uses the exact multi-pass route over the whole row
+  uint32_t ticket_hist;   // blocks of the current histogram pass that have finished this row
+  uint32_t ticket_count;  // blocks of the count pass that have finished this row
+  uint32_t pad[6];
 };
 
 // Byte offsets of the workspace regions; computed identically for sizing and use.
@@ -120,7 +123,7 @@ cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t 
 cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     cudaStream_t st);
+                                     uint32_t* hdr, uint32_t* hist, cudaStream_t st);
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,

@@ -27,9 +27,13 @@ __device__ __forceinline__ uint32_t mix32(uint32_t v) {   // integer finaliser, 
 constexpr int kChunk = 32;
 constexpr int kSampleUnroll = 8;
 
+// The kernel also resets the row's selection state, its radix histogram and (block 0) the
+// status words, so that no separate initialisation launch is needed on this route.
 __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 RowState* __restrict__ rows, uint32_t n_sample,
-                                                                uint32_t stride, uint32_t j_rank) {
+                                                                uint32_t stride, uint32_t j_rank, uint32_t K,
+                                                                uint32_t* __restrict__ hdr,
+                                                                uint32_t* __restrict__ hist) {
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
   __shared__ uint32_t s_pick[2];
@@ -37,6 +41,13 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   const uint32_t row = blockIdx.x;
   const uint32_t* rowp = gbits + (uint64_t)row * d;
 
+  if (blockIdx.x == 0 && tid < (uint32_t)kHdrWords) hdr[tid] = 0u;
+  if (tid == 0) {
+    RowState rs = {};
+    rs.k_rem = K;
+    rows[row] = rs;                                // tau_lo is filled in at the end
+  }
+  for (uint32_t b = tid; b < (uint32_t)kHistBins; b += 1024) hist[(uint64_t)row * kHistBins + b] = 0u;
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
   __syncthreads();
   if (stride == 0) {                              // short row: every entry is inspected
@@ -168,13 +179,14 @@ __global__ void __launch_bounds__(kTileThreads) filter_kernel(const uint32_t* __
 }  // namespace
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     cudaStream_t st) {
+                                     uint32_t* hdr, uint32_t* hist, cudaStream_t st) {
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
   cudaError_t e = cudaFuncSetAttribute(sample_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  sample_threshold_kernel<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank);
+  sample_threshold_kernel<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
+                                                   (uint32_t)L.K, hdr, hist);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   prof_mark(kPhaseSampled, st);

@@ -7,15 +7,18 @@
 //   * candidates: the filtered list of a row (few entries, L2 resident) -- normal case;
 //   * whole row:  every entry of the row -- for large K, and for rows whose filter
 //                 produced fewer than K or more than `cap` survivors.
-// Each kernel decides per row which source is live (row_uses_candidates), so the
-// host never has to look at device state.
+// Each launch carries blocks for both sources; a block looks at its row's state and
+// works only if its source is the live one (row_uses_candidates), so the host never
+// has to look at device state.  The per-row follow-up of a pass (choosing the digit,
+// scanning the per-tile counts) is done by whichever block finishes that row last.
 #include "s3gd_tile.cuh"
 
 namespace s3gd {
 
 namespace {
 
-constexpr int kHistThreads = 256;
+constexpr int kSelThreads = 256;
+static_assert(kSelThreads == kTileThreads, "row-source blocks load tiles with kTileThreads threads");
 
 // ---------------------------------------------------------------- init
 __global__ void init_kernel(uint32_t* __restrict__ hdr, RowState* __restrict__ rows, uint32_t* __restrict__ hist,
@@ -23,12 +26,28 @@ __global__ void init_kernel(uint32_t* __restrict__ hdr, RowState* __restrict__ r
   const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
   if (tid < (uint32_t)kHdrWords) hdr[tid] = 0u;
   for (uint32_t m = tid; m < (uint32_t)M; m += nthr) {
-    RowState rs;
-    rs.tau_lo = 0u; rs.n_cand = 0u; rs.prefix = 0u; rs.k_rem = K;
-    rs.tau = 0u; rs.take_ties = 0u; rs.n_emitted = 0u; rs.exact = force_exact;
+    RowState rs = {};
+    rs.k_rem = K;
+    rs.exact = force_exact;
     rows[m] = rs;
   }
   for (uint64_t i = tid; i < (uint64_t)M * kHistBins; i += nthr) hist[i] = 0u;
+}
+
+// True in exactly one block per row: the one that arrives after all others of that row have
+// published their global writes.  Every block of the row must call it exactly once.
+__device__ __forceinline__ bool last_block_of_row(uint32_t* ticket, uint32_t n_blocks, uint32_t* s_flag) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t t = atomicAdd(ticket, 1u);
+    *s_flag = (t == n_blocks - 1u) ? 1u : 0u;
+    if (t == n_blocks - 1u) atomicExch(ticket, 0u);      // ready for the next pass
+  }
+  __syncthreads();
+  const bool last = *s_flag != 0u;
+  if (last) __threadfence();
+  return last;
 }
 
 // ------------------------------------------------------- histogram passes
@@ -43,99 +62,26 @@ __device__ __forceinline__ bool in_prefix(uint32_t key, uint32_t prefix, int pas
   return pass == 0 || (key >> pass_shift(pass - 1)) == prefix;
 }
 
-__device__ __forceinline__ void hist_flush(const uint32_t* s_hist, uint32_t* __restrict__ g_hist, int nbins) {
-  for (int b = threadIdx.x; b < nbins; b += blockDim.x) {
-    uint32_t c = s_hist[b];
-    if (c) atomicAdd(&g_hist[b], c);
-  }
-}
-
-// grid (blocks per row, M)
-__global__ void __launch_bounds__(kHistThreads) hist_cand_kernel(const uint2* __restrict__ cand, uint32_t cap,
-                                                                 const RowState* __restrict__ rows, uint32_t K,
-                                                                 uint32_t* __restrict__ hist, int pass) {
-  __shared__ uint32_t s_hist[kHistBins];
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (!row_uses_candidates(rs, K, cap)) return;
-  const uint32_t n = rs.n_cand;
-  if ((uint64_t)blockIdx.x * kHistThreads >= n) return;
+// Find the digit in which the k_rem-th largest entry lies, fix it, and clear the
+// histogram for the next pass.  One block of kSelThreads threads.
+__device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t row, uint32_t* __restrict__ h,
+                                           uint32_t* __restrict__ hdr, int pass, uint32_t* s_sum, uint32_t* s_sel) {
+  const uint32_t tid = threadIdx.x;
   const int nbins = 1 << pass_bits(pass);
-  for (int b = threadIdx.x; b < nbins; b += kHistThreads) s_hist[b] = 0u;
-  __syncthreads();
-  const uint2* c = cand + (uint64_t)row * cap;
-  const uint32_t step = gridDim.x * kHistThreads;
-  const uint32_t n_round = (n + 31u) & ~31u;          // whole warps stay in the loop together
-  for (uint32_t i = blockIdx.x * kHistThreads + threadIdx.x; i < n_round; i += step) {
-    bool on = i < n;
-    uint32_t key = on ? (c[i].x & kAbsMask) : 0u;
-    on = on && in_prefix(key, rs.prefix, pass);
-    hist_add(s_hist, on, (key >> pass_shift(pass)) & (uint32_t)(nbins - 1));
-  }
-  __syncthreads();
-  hist_flush(s_hist, hist + (uint64_t)row * kHistBins, nbins);
-}
-
-// grid (blocks per row, M); each block walks tiles of its row
-__global__ void __launch_bounds__(kTileThreads) hist_row_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                                uint32_t n_tiles, uint32_t cap,
-                                                                const RowState* __restrict__ rows, uint32_t K,
-                                                                uint32_t* __restrict__ hist, int pass) {
-  __shared__ uint32_t s_hist[kHistBins];
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (row_uses_candidates(rs, K, cap)) return;
-  const int nbins = 1 << pass_bits(pass);
-  for (int b = threadIdx.x; b < nbins; b += kTileThreads) s_hist[b] = 0u;
-  __syncthreads();
-  const uint32_t* rowp = gbits + (uint64_t)row * d;
-  const uint32_t head = row_head(rowp, d);
-  const uint32_t mask = (uint32_t)(nbins - 1);
-  for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-    Tile T;
-    load_tile(T, rowp, d, head, t);
-    if (t == 0 && threadIdx.x < 32) {
-      uint32_t key = T.head_bits & kAbsMask;
-      hist_add(s_hist, T.head_valid && in_prefix(key, rs.prefix, pass), (key >> pass_shift(pass)) & mask);
-    }
-#pragma unroll
-    for (int it = 0; it < kTileIters; ++it) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t key = T.bits[it][q] & kAbsMask;
-        bool on = (T.valid[it] >> q & 1u) && in_prefix(key, rs.prefix, pass);
-        hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
-      }
-    }
-  }
-  __syncthreads();
-  hist_flush(s_hist, hist + (uint64_t)row * kHistBins, nbins);
-}
-
-// One CTA per row: find the digit in which the k_rem-th largest entry lies, fix it,
-// and clear the histogram for the next pass.
-__global__ void __launch_bounds__(256) pick_kernel(RowState* __restrict__ rows, uint32_t* __restrict__ hist,
-                                                   uint32_t* __restrict__ hdr, int pass) {
-  __shared__ uint32_t s_sum[256];
-  __shared__ uint32_t s_sel[2];
-  const uint32_t row = blockIdx.x, tid = threadIdx.x;
-  const int nbins = 1 << pass_bits(pass);
-  const int per = nbins / 256;                       // 8 or 4 bins per thread, ascending
-  uint32_t* h = hist + (uint64_t)row * kHistBins;
+  const int per = nbins / kSelThreads;               // 8 or 4 bins per thread, ascending
   uint32_t c[8];
   uint32_t mine = 0;
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    c[i] = (i < per) ? h[tid * per + i] : 0u;
+    c[i] = (i < per) ? __ldcg(h + tid * per + i) : 0u;
     mine += c[i];
   }
   s_sum[tid] = mine;
   if (tid == 0) { s_sel[0] = 0xFFFFFFFFu; s_sel[1] = 0u; }
   __syncthreads();
   const uint32_t k_rem = rows[row].k_rem;
-  // entries in bins owned by higher threads
-  uint32_t above = 0;
-  for (int t = 255; t > (int)tid; --t) above += s_sum[t];
+  uint32_t above = 0;                                // entries in bins owned by higher threads
+  for (int t = kSelThreads - 1; t > (int)tid; --t) above += s_sum[t];
   if (above < k_rem && above + mine >= k_rem) {      // exactly one thread
     uint32_t a = above;
     for (int i = per - 1; i >= 0; --i) {
@@ -147,19 +93,85 @@ __global__ void __launch_bounds__(256) pick_kernel(RowState* __restrict__ rows, 
   for (int i = 0; i < per; ++i) h[tid * per + i] = 0u;
   if (tid == 0) {
     uint32_t digit = s_sel[0], a = s_sel[1];
-    RowState rs = rows[row];
     if (digit == 0xFFFFFFFFu) {                      // fewer than k_rem entries: cannot happen for a valid row
       atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
       digit = 0u; a = 0u;
     }
-    rs.prefix = (rs.prefix << pass_bits(pass)) | digit;
-    rs.k_rem = k_rem - a;
+    const uint32_t prefix = (rows[row].prefix << pass_bits(pass)) | digit;
+    rows[row].prefix = prefix;
+    rows[row].k_rem = k_rem - a;
     if (pass == kNumPasses - 1) {
-      rs.tau = rs.prefix;
-      rs.take_ties = rs.k_rem;
+      rows[row].tau = prefix;
+      rows[row].take_ties = k_rem - a;
     }
-    rows[row] = rs;
   }
+}
+
+// grid (gx_c + gx_r, M): the first gx_c blocks of a row walk its candidates, the others its tiles.
+__global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                                uint32_t cap, RowState* __restrict__ rows, uint32_t K,
+                                                                uint32_t* __restrict__ hist,
+                                                                uint32_t* __restrict__ hdr, int pass, uint32_t gx_c) {
+  __shared__ uint32_t s_hist[kHistBins];
+  __shared__ uint32_t s_sum[kSelThreads];
+  __shared__ uint32_t s_sel[2];
+  __shared__ uint32_t s_flag;
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  const bool use_c = row_uses_candidates(rs, K, cap);
+  const bool is_c = blockIdx.x < gx_c;
+  const int nbins = 1 << pass_bits(pass);
+  const uint32_t mask = (uint32_t)(nbins - 1);
+  uint32_t* g_hist = hist + (uint64_t)row * kHistBins;
+  bool worked = false;
+  if (is_c && use_c && (uint64_t)blockIdx.x * kSelThreads < rs.n_cand) {
+    worked = true;
+    for (int b = threadIdx.x; b < nbins; b += kSelThreads) s_hist[b] = 0u;
+    __syncthreads();
+    const uint2* c = cand + (uint64_t)row * cap;
+    const uint32_t n = rs.n_cand, step = gx_c * kSelThreads;
+    const uint32_t n_round = (n + 31u) & ~31u;        // whole warps stay in the loop together
+    for (uint32_t i = blockIdx.x * kSelThreads + threadIdx.x; i < n_round; i += step) {
+      bool on = i < n;
+      const uint32_t key = on ? (c[i].x & kAbsMask) : 0u;
+      on = on && in_prefix(key, rs.prefix, pass);
+      hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
+    }
+  } else if (!is_c && !use_c) {
+    worked = true;
+    for (int b = threadIdx.x; b < nbins; b += kSelThreads) s_hist[b] = 0u;
+    __syncthreads();
+    const uint32_t* rowp = gbits + (uint64_t)row * d;
+    const uint32_t head = row_head(rowp, d);
+    const uint32_t gx_r = gridDim.x - gx_c;
+    for (uint32_t t = blockIdx.x - gx_c; t < n_tiles; t += gx_r) {
+      Tile T;
+      load_tile(T, rowp, d, head, t);
+      if (t == 0 && threadIdx.x < 32) {
+        const uint32_t key = T.head_bits & kAbsMask;
+        hist_add(s_hist, T.head_valid && in_prefix(key, rs.prefix, pass), (key >> pass_shift(pass)) & mask);
+      }
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t key = T.bits[it][q] & kAbsMask;
+          const bool on = (T.valid[it] >> q & 1u) && in_prefix(key, rs.prefix, pass);
+          hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
+        }
+      }
+    }
+  }
+  if (worked) {
+    __syncthreads();
+    for (int b = threadIdx.x; b < nbins; b += kSelThreads) {
+      const uint32_t c = s_hist[b];
+      if (c) atomicAdd(&g_hist[b], c);
+    }
+  }
+  if (last_block_of_row(&rows[row].ticket_hist, gridDim.x, &s_flag))
+    pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel);
 }
 
 }  // namespace

@@ -1,27 +1,23 @@
-// Second half of s3gd_select.cu: per-tile counts, their scan, the ordered emission
+// Second half of s3gd_select.cu: per-tile counts and their scan, the ordered emission,
 // and the host-side sequencing of the whole selection.
 namespace s3gd {
 namespace {
 
 // ------------------------------------------------------------ per-tile counts
-// cnt[row][tile] = (#entries above tau, #entries equal to tau) in that tile
+// cnt[row][tile] = (#entries above tau, #entries equal to tau) in that tile.
 // candidates: one warp per tile segment
-__global__ void __launch_bounds__(256) count_cand_kernel(const uint2* __restrict__ cand, uint32_t cap,
-                                                         const uint2* __restrict__ seg, uint32_t n_tiles,
-                                                         const RowState* __restrict__ rows, uint32_t K,
-                                                         uint2* __restrict__ cnt) {
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (!row_uses_candidates(rs, K, cap)) return;
+__device__ __forceinline__ void count_cand(const uint2* __restrict__ cand, uint32_t cap, const uint2* __restrict__ seg,
+                                           uint32_t n_tiles, const RowState& rs, uint32_t row, uint32_t bx,
+                                           uint32_t gx, uint2* __restrict__ cnt) {
   const uint32_t lane = threadIdx.x & 31;
-  const uint32_t warps = gridDim.x * (blockDim.x >> 5);
+  const uint32_t warps = gx * (kSelThreads >> 5);
   const uint2* c = cand + (uint64_t)row * cap;
-  for (uint32_t t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
+  for (uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
     const uint2 sg = seg[(uint64_t)row * n_tiles + t];
     uint32_t gt = 0, eq = 0;
     for (uint32_t i0 = 0; i0 < sg.y; i0 += 32) {
-      uint32_t i = i0 + lane;
-      uint32_t key = (i < sg.y) ? (c[sg.x + i].x & kAbsMask) : 0u;
+      const uint32_t i = i0 + lane;
+      const uint32_t key = (i < sg.y) ? (c[sg.x + i].x & kAbsMask) : 0u;
       gt += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key > rs.tau));
       eq += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key == rs.tau));
     }
@@ -30,31 +26,26 @@ __global__ void __launch_bounds__(256) count_cand_kernel(const uint2* __restrict
 }
 
 // whole row: one CTA per tile
-__global__ void __launch_bounds__(kTileThreads) count_row_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                                 uint32_t n_tiles, uint32_t cap,
-                                                                 const RowState* __restrict__ rows, uint32_t K,
-                                                                 uint2* __restrict__ cnt) {
-  __shared__ uint32_t s_gt[kWarpsPerTile], s_eq[kWarpsPerTile];
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (row_uses_candidates(rs, K, cap)) return;
+__device__ __forceinline__ void count_row(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
+                                          const RowState& rs, uint32_t row, uint32_t bx, uint32_t gx,
+                                          uint2* __restrict__ cnt, uint32_t* s_gt, uint32_t* s_eq) {
   const uint32_t* rowp = gbits + (uint64_t)row * d;
   const uint32_t head = row_head(rowp, d);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+  for (uint32_t t = bx; t < n_tiles; t += gx) {
     Tile T;
     load_tile(T, rowp, d, head, t);
     uint32_t gt = 0, eq = 0;
     if (T.head_valid) {
-      uint32_t key = T.head_bits & kAbsMask;
+      const uint32_t key = T.head_bits & kAbsMask;
       gt += key > rs.tau; eq += key == rs.tau;
     }
 #pragma unroll
     for (int it = 0; it < kTileIters; ++it) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        uint32_t key = T.bits[it][q] & kAbsMask;
-        uint32_t ok = T.valid[it] >> q & 1u;
+        const uint32_t key = T.bits[it][q] & kAbsMask;
+        const uint32_t ok = T.valid[it] >> q & 1u;
         gt += ok & (uint32_t)(key > rs.tau);
         eq += ok & (uint32_t)(key == rs.tau);
       }
@@ -76,24 +67,25 @@ __global__ void __launch_bounds__(kTileThreads) count_row_kernel(const uint32_t*
 }
 
 // ------------------------------------------------------------------- scan
-// One CTA per row.  In: cnt[tile] = (gt, eq).  Out, in place: (first output position of
-// the tile, number of entries equal to tau in earlier tiles).  A tile keeps all its
-// entries above tau, and of its entries equal to tau those whose running number
-// (in index order over the whole row) is below take_ties.
-__device__ __forceinline__ uint32_t block_exclusive_scan_1024(uint32_t v, uint32_t* s_warp, uint32_t* total) {
+// One block per row (the last one to finish counting).  In: cnt[tile] = (gt, eq).  Out, in
+// place: (first output position of the tile, number of entries equal to tau in earlier
+// tiles).  A tile keeps all its entries above tau, and of its entries equal to tau those
+// whose running number (in index order over the whole row) is below take_ties.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s_warp, uint32_t* total) {
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t inc = v;
 #pragma unroll
   for (int s = 1; s < 32; s <<= 1) {
-    uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, s);
+    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, s);
     if (lane >= (uint32_t)s) inc += o;
   }
   __syncthreads();
   if (lane == 31) s_warp[warp] = inc;
   __syncthreads();
   uint32_t off = 0, tot = 0;
-  for (int w = 0; w < 32; ++w) {
-    uint32_t c = s_warp[w];
+#pragma unroll
+  for (int w = 0; w < kSelThreads / 32; ++w) {
+    const uint32_t c = s_warp[w];
     if ((uint32_t)w < warp) off += c;
     tot += c;
   }
@@ -101,39 +93,37 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_1024(uint32_t v, uint32
   return off + inc - v;
 }
 
-__global__ void __launch_bounds__(1024) scan_kernel(uint2* __restrict__ cnt, uint32_t n_tiles,
-                                                    RowState* __restrict__ rows, uint32_t K, uint32_t cap,
-                                                    uint32_t* __restrict__ hdr) {
-  __shared__ uint32_t s_warp[32];
-  const uint32_t row = blockIdx.x, tid = threadIdx.x;
-  uint2* c = cnt + (uint64_t)row * n_tiles;
+__device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles, RowState* __restrict__ rows,
+                                         uint32_t row, uint32_t K, uint32_t cap, uint32_t* __restrict__ hdr,
+                                         uint32_t* s_warp) {
+  const uint32_t tid = threadIdx.x;
   const uint32_t take = rows[row].take_ties;
-  const uint32_t per = (n_tiles + 1023u) / 1024u;
+  const uint32_t per = (n_tiles + kSelThreads - 1) / kSelThreads;
   const uint32_t lo = tid * per < n_tiles ? tid * per : n_tiles;
   const uint32_t hi = lo + per < n_tiles ? lo + per : n_tiles;
   uint32_t eq_sum = 0;
-  for (uint32_t t = lo; t < hi; ++t) eq_sum += c[t].y;
+  for (uint32_t t = lo; t < hi; ++t) eq_sum += __ldcg(&c[t]).y;
   uint32_t tot_eq;
-  const uint32_t eq_before = block_exclusive_scan_1024(eq_sum, s_warp, &tot_eq);
+  const uint32_t eq_before = block_exclusive_scan(eq_sum, s_warp, &tot_eq);
   uint32_t sel_sum = 0, run_eq = eq_before;
   for (uint32_t t = lo; t < hi; ++t) {
-    uint2 v = c[t];
-    uint32_t room = run_eq < take ? take - run_eq : 0u;
+    const uint2 v = __ldcg(&c[t]);
+    const uint32_t room = run_eq < take ? take - run_eq : 0u;
     sel_sum += v.x + (v.y < room ? v.y : room);
     run_eq += v.y;
   }
   uint32_t tot_sel;
-  uint32_t out = block_exclusive_scan_1024(sel_sum, s_warp, &tot_sel);
+  uint32_t out = block_exclusive_scan(sel_sum, s_warp, &tot_sel);
   run_eq = eq_before;
   for (uint32_t t = lo; t < hi; ++t) {
-    uint2 v = c[t];
-    uint32_t room = run_eq < take ? take - run_eq : 0u;
+    const uint2 v = __ldcg(&c[t]);
+    const uint32_t room = run_eq < take ? take - run_eq : 0u;
     c[t] = make_uint2(out, run_eq);
     out += v.x + (v.y < room ? v.y : room);
     run_eq += v.y;
   }
   if (tid == 0) {
-    RowState rs = rows[row];
+    const RowState rs = rows[row];
     rows[row].n_emitted = tot_sel;
     if (tot_sel != K) {
       atomicAdd(hdr + kHdrBadCount, 1u);
@@ -142,6 +132,25 @@ __global__ void __launch_bounds__(1024) scan_kernel(uint2* __restrict__ cnt, uin
     if (!row_uses_candidates(rs, K, cap)) atomicAdd(hdr + kHdrExactRows, 1u);
     atomicMax(hdr + kHdrMaxCand, rs.n_cand);
   }
+}
+
+// grid (gx_c + gx_r, M)
+__global__ void __launch_bounds__(kSelThreads) count_scan_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                 uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                                 uint32_t cap, const uint2* __restrict__ seg,
+                                                                 RowState* __restrict__ rows, uint32_t K,
+                                                                 uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
+                                                                 uint32_t gx_c) {
+  __shared__ uint32_t s_gt[kWarpsPerTile], s_eq[kWarpsPerTile], s_warp[kSelThreads / 32];
+  __shared__ uint32_t s_flag;
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  const bool use_c = row_uses_candidates(rs, K, cap);
+  const bool is_c = blockIdx.x < gx_c;
+  if (is_c && use_c) count_cand(cand, cap, seg, n_tiles, rs, row, blockIdx.x, gx_c, cnt);
+  else if (!is_c && !use_c) count_row(gbits, d, n_tiles, rs, row, blockIdx.x - gx_c, gridDim.x - gx_c, cnt, s_gt, s_eq);
+  if (last_block_of_row(&rows[row].ticket_count, gridDim.x, &s_flag))
+    scan_row(cnt + (uint64_t)row * n_tiles, n_tiles, rows, row, K, cap, hdr, s_warp);
 }
 
 // ------------------------------------------------------------------- emit
@@ -155,17 +164,13 @@ struct EmitOut {
 // candidates: one warp per tile segment, 32 entries per step.  Sign bits of the (at most
 // two) output words a step touches are gathered with a warp OR-reduction and merged
 // into the zeroed output with one atomic per word.
-__global__ void __launch_bounds__(256) emit_cand_kernel(const uint2* __restrict__ cand, uint32_t cap,
-                                                        const uint2* __restrict__ seg,
-                                                        const uint2* __restrict__ scan, uint32_t n_tiles,
-                                                        const RowState* __restrict__ rows, EmitOut o) {
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (!row_uses_candidates(rs, o.K, cap)) return;
+__device__ __forceinline__ void emit_cand(const uint2* __restrict__ cand, uint32_t cap, const uint2* __restrict__ seg,
+                                          const uint2* __restrict__ scan, uint32_t n_tiles, const RowState& rs,
+                                          uint32_t row, uint32_t bx, uint32_t gx, const EmitOut& o) {
   const uint32_t lane = threadIdx.x & 31, lt = lanemask_lt();
-  const uint32_t warps = gridDim.x * (blockDim.x >> 5);
+  const uint32_t warps = gx * (kSelThreads >> 5);
   const uint2* c = cand + (uint64_t)row * cap;
-  for (uint32_t t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
+  for (uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
     const uint2 sg = seg[(uint64_t)row * n_tiles + t];
     if (sg.y == 0) continue;
     const uint2 sc = scan[(uint64_t)row * n_tiles + t];
@@ -202,18 +207,13 @@ __global__ void __launch_bounds__(256) emit_cand_kernel(const uint2* __restrict_
 }
 
 // whole row: one CTA per tile; two ordered rankings (ties, then kept entries)
-__global__ void __launch_bounds__(kTileThreads) emit_row_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                                uint32_t n_tiles, uint32_t cap,
-                                                                const uint2* __restrict__ scan,
-                                                                const RowState* __restrict__ rows, EmitOut o) {
-  __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
-  if (row_uses_candidates(rs, o.K, cap)) return;
+__device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
+                                         const uint2* __restrict__ scan, const RowState& rs, uint32_t row,
+                                         uint32_t bx, uint32_t gx, const EmitOut& o, uint32_t* s_wtot) {
   const uint32_t* rowp = gbits + (uint64_t)row * d;
   const uint32_t head = row_head(rowp, d);
   const uint32_t lane = threadIdx.x & 31;
-  for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+  for (uint32_t t = bx; t < n_tiles; t += gx) {
     const uint2 sc = scan[(uint64_t)row * n_tiles + t];
     Tile T;
     load_tile(T, rowp, d, head, t);
@@ -293,6 +293,22 @@ __global__ void __launch_bounds__(kTileThreads) emit_row_kernel(const uint32_t* 
   }
 }
 
+// grid (gx_c + gx_r, M)
+__global__ void __launch_bounds__(kSelThreads) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                           uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                           uint32_t cap, const uint2* __restrict__ seg,
+                                                           const uint2* __restrict__ scan,
+                                                           const RowState* __restrict__ rows, EmitOut o,
+                                                           uint32_t gx_c) {
+  __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
+  const uint32_t row = blockIdx.y;
+  const RowState rs = rows[row];
+  const bool use_c = row_uses_candidates(rs, o.K, cap);
+  const bool is_c = blockIdx.x < gx_c;
+  if (is_c && use_c) emit_cand(cand, cap, seg, scan, n_tiles, rs, row, blockIdx.x, gx_c, o);
+  else if (!is_c && !use_c) emit_row(gbits, d, n_tiles, scan, rs, row, blockIdx.x - gx_c, gridDim.x - gx_c, o, s_wtot);
+}
+
 inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)(v < lo ? lo : (v > hi ? hi : v)); }
 
 }  // namespace
@@ -317,47 +333,35 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     count_launch();                                 \
   } while (0)
 
-  init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K,
-                                                                                           use_filter ? 0u : 1u);
-  S3GD_CHECK_LAUNCH();
   if (use_filter) {
-    cudaError_t e = launch_sample_and_filter(gbits, L, rows, cand, seg, st);
+    cudaError_t e = launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, st);
     if (e != cudaSuccess) return e;
   } else {
+    init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
+    S3GD_CHECK_LAUNCH();
     prof_mark(kPhaseSampled, st);
   }
   prof_mark(kPhaseFiltered, st);
-  // blocks per row for the passes over candidates / over whole rows
-  const dim3 grid_c(clampu(((uint64_t)L.cap + 4095) / 4096, 1, 64), M);
-  const dim3 grid_r(clampu(L.n_tiles, 1, ((uint64_t)kSMs * 8 + M - 1) / M), M);
-  const dim3 grid_w(clampu(((uint64_t)L.n_tiles + 7) / 8, 1, ((uint64_t)kSMs * 8 + M - 1) / M), M);
+  // blocks per row: for the passes over candidates (hist: 4096 entries per block; count/emit:
+  // 8 tile segments per block) and for the passes over whole rows
+  const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * 8 + M - 1) / M);
+  const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, 64) : 0u;
+  const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
+  const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
   for (int pass = 0; pass < kNumPasses; ++pass) {
-    if (use_filter) {
-      hist_cand_kernel<<<grid_c, kHistThreads, 0, st>>>(cand, L.cap, rows, K, hist, pass);
-      S3GD_CHECK_LAUNCH();
-    }
-    hist_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, rows, K, hist, pass);
-    S3GD_CHECK_LAUNCH();
-    pick_kernel<<<M, 256, 0, st>>>(rows, hist, hdr, pass);
+    hist_pick_kernel<<<dim3(gx_hist_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, rows, K,
+                                                                        hist, hdr, pass, gx_hist_c);
     S3GD_CHECK_LAUNCH();
   }
   prof_mark(kPhaseThreshold, st);
-  if (use_filter) {
-    count_cand_kernel<<<grid_w, 256, 0, st>>>(cand, L.cap, seg, L.n_tiles, rows, K, cnt);
-    S3GD_CHECK_LAUNCH();
-  }
-  count_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, rows, K, cnt);
-  S3GD_CHECK_LAUNCH();
-  scan_kernel<<<M, 1024, 0, st>>>(cnt, L.n_tiles, rows, K, L.cap, hdr);
+  count_scan_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows,
+                                                                       K, cnt, hdr, gx_tile_c);
   S3GD_CHECK_LAUNCH();
   EmitOut o;
   o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
   o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
-  if (use_filter) {
-    emit_cand_kernel<<<grid_w, 256, 0, st>>>(cand, L.cap, seg, cnt, L.n_tiles, rows, o);
-    S3GD_CHECK_LAUNCH();
-  }
-  emit_row_kernel<<<grid_r, kTileThreads, 0, st>>>(gbits, L.d, L.n_tiles, L.cap, cnt, rows, o);
+  emit_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
+                                                                 gx_tile_c);
   S3GD_CHECK_LAUNCH();
 #undef S3GD_CHECK_LAUNCH
   prof_mark(kPhaseEmitted, st);
