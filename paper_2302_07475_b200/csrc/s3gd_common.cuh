@@ -51,7 +51,8 @@ struct RowState {
   uint32_t exact;      // 1: this row uses the exact multi-pass route over the whole row
   uint32_t ticket_hist;   // blocks of the current histogram pass that have finished this row
   uint32_t ticket_count;  // blocks of the count pass that have finished this row
-  uint32_t pad[6];
+  uint32_t done;          // 1: the single-CTA selection has already finished this row
+  uint32_t pad[5];
 };
 
 // Byte offsets of the workspace regions; computed identically for sizing and use.
@@ -101,6 +102,12 @@ __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
 __device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
   return rs.exact == 0u && rs.n_cand >= K && rs.n_cand <= cap;
 }
+// Shared memory the single-CTA selection needs for a row: the candidates' bit patterns and two
+// 8-byte tables per tile.  Rows that fit are finished by that kernel; the others by the general passes.
+constexpr uint32_t kSmallSelectBytes = 212 * 1024;
+__host__ __device__ __forceinline__ bool fits_single_cta(uint32_t n_cand, uint32_t n_tiles) {
+  return (uint64_t)n_cand * 4u + (uint64_t)n_tiles * 16u <= kSmallSelectBytes;
+}
 #endif
 
 // ------------------------------------------------------------------ profiling
@@ -124,6 +131,14 @@ cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
                                      uint32_t* hdr, uint32_t* hist, cudaStream_t st);
+struct EmitOut {
+  uint32_t* idx;        // [M x K] or NULL
+  uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
+  int32_t* counter;     // [d] or NULL
+  uint32_t K, words;
+};
+cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* cand, const uint2* seg, uint32_t* hdr,
+                                const EmitOut& o, cudaStream_t st);
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,

@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* 
   __shared__ uint32_t s_flag;
   const uint32_t row = blockIdx.y;
   const RowState rs = rows[row];
+  if (rs.done) return;                               // finished by the single-CTA selection (all blocks of the row agree)
   const bool use_c = row_uses_candidates(rs, K, cap);
   const bool is_c = blockIdx.x < gx_c;
   const int nbins = 1 << pass_bits(pass);

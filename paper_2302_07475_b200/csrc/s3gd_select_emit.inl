@@ -98,34 +98,26 @@ __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles
                                          uint32_t* s_warp) {
   const uint32_t tid = threadIdx.x;
   const uint32_t take = rows[row].take_ties;
-  const uint32_t per = (n_tiles + kSelThreads - 1) / kSelThreads;
-  const uint32_t lo = tid * per < n_tiles ? tid * per : n_tiles;
-  const uint32_t hi = lo + per < n_tiles ? lo + per : n_tiles;
-  uint32_t eq_sum = 0;
-  for (uint32_t t = lo; t < hi; ++t) eq_sum += __ldcg(&c[t]).y;
-  uint32_t tot_eq;
-  const uint32_t eq_before = block_exclusive_scan(eq_sum, s_warp, &tot_eq);
-  uint32_t sel_sum = 0, run_eq = eq_before;
-  for (uint32_t t = lo; t < hi; ++t) {
-    const uint2 v = __ldcg(&c[t]);
+  uint32_t carry_eq = 0, carry_out = 0;
+  uint2 next = tid < n_tiles ? __ldcg(&c[tid]) : make_uint2(0u, 0u);
+  for (uint32_t base = 0; base < n_tiles; base += kSelThreads) {     // kSelThreads tiles per round, next round in flight
+    const uint32_t t = base + tid;
+    const uint2 v = next;
+    const uint32_t tn = t + kSelThreads;
+    next = tn < n_tiles ? __ldcg(&c[tn]) : make_uint2(0u, 0u);
+    uint32_t tot_eq, tot_sel;
+    const uint32_t run_eq = carry_eq + block_exclusive_scan(v.y, s_warp, &tot_eq);
     const uint32_t room = run_eq < take ? take - run_eq : 0u;
-    sel_sum += v.x + (v.y < room ? v.y : room);
-    run_eq += v.y;
-  }
-  uint32_t tot_sel;
-  uint32_t out = block_exclusive_scan(sel_sum, s_warp, &tot_sel);
-  run_eq = eq_before;
-  for (uint32_t t = lo; t < hi; ++t) {
-    const uint2 v = __ldcg(&c[t]);
-    const uint32_t room = run_eq < take ? take - run_eq : 0u;
-    c[t] = make_uint2(out, run_eq);
-    out += v.x + (v.y < room ? v.y : room);
-    run_eq += v.y;
+    const uint32_t sel = v.x + (v.y < room ? v.y : room);
+    const uint32_t out = carry_out + block_exclusive_scan(sel, s_warp, &tot_sel);
+    if (t < n_tiles) c[t] = make_uint2(out, run_eq);
+    carry_eq += tot_eq;
+    carry_out += tot_sel;
   }
   if (tid == 0) {
     const RowState rs = rows[row];
-    rows[row].n_emitted = tot_sel;
-    if (tot_sel != K) {
+    rows[row].n_emitted = carry_out;
+    if (carry_out != K) {
       atomicAdd(hdr + kHdrBadCount, 1u);
       atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
     }
@@ -145,6 +137,7 @@ __global__ void __launch_bounds__(kSelThreads) count_scan_kernel(const uint32_t*
   __shared__ uint32_t s_flag;
   const uint32_t row = blockIdx.y;
   const RowState rs = rows[row];
+  if (rs.done) return;
   const bool use_c = row_uses_candidates(rs, K, cap);
   const bool is_c = blockIdx.x < gx_c;
   if (is_c && use_c) count_cand(cand, cap, seg, n_tiles, rs, row, blockIdx.x, gx_c, cnt);
@@ -154,12 +147,6 @@ __global__ void __launch_bounds__(kSelThreads) count_scan_kernel(const uint32_t*
 }
 
 // ------------------------------------------------------------------- emit
-struct EmitOut {
-  uint32_t* idx;        // [M x K] or NULL
-  uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
-  int32_t* counter;     // [d] or NULL
-  uint32_t K, words;
-};
 
 // candidates: one warp per tile segment, 32 entries per step.  Sign bits of the (at most
 // two) output words a step touches are gathered with a warp OR-reduction and merged
@@ -303,6 +290,7 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(const uint32_t* __res
   __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
   const uint32_t row = blockIdx.y;
   const RowState rs = rows[row];
+  if (rs.done) return;
   const bool use_c = row_uses_candidates(rs, o.K, cap);
   const bool is_c = blockIdx.x < gx_c;
   if (is_c && use_c) emit_cand(cand, cap, seg, scan, n_tiles, rs, row, blockIdx.x, gx_c, o);
@@ -342,6 +330,13 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     prof_mark(kPhaseSampled, st);
   }
   prof_mark(kPhaseFiltered, st);
+  EmitOut o;
+  o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
+  o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
+  if (use_filter) {                                  // rows whose candidates fit one SM are finished here
+    cudaError_t e = launch_select_small(L, rows, cand, seg, hdr, o, st);
+    if (e != cudaSuccess) return e;
+  }
   // blocks per row: for the passes over candidates (hist: 4096 entries per block; count/emit:
   // 8 tile segments per block) and for the passes over whole rows
   const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * 8 + M - 1) / M);
@@ -357,9 +352,6 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   count_scan_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows,
                                                                        K, cnt, hdr, gx_tile_c);
   S3GD_CHECK_LAUNCH();
-  EmitOut o;
-  o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
-  o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
   emit_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
                                                                  gx_tile_c);
   S3GD_CHECK_LAUNCH();
