@@ -102,11 +102,11 @@ __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
 __device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
   return rs.exact == 0u && rs.n_cand >= K && rs.n_cand <= cap;
 }
-// Shared memory the single-CTA selection needs for a row: the candidates' bit patterns and two
-// 8-byte tables per tile.  Rows that fit are finished by that kernel; the others by the general passes.
+// Shared memory the single-CTA selection needs for a row: bit pattern and index of every
+// candidate.  Rows that fit are finished by that kernel; the others by the general passes.
 constexpr uint32_t kSmallSelectBytes = 212 * 1024;
-__host__ __device__ __forceinline__ bool fits_single_cta(uint32_t n_cand, uint32_t n_tiles) {
-  return (uint64_t)n_cand * 4u + (uint64_t)n_tiles * 16u <= kSmallSelectBytes;
+__host__ __device__ __forceinline__ bool fits_single_cta(uint32_t n_cand) {
+  return (uint64_t)n_cand * 8u <= kSmallSelectBytes;
 }
 #endif
 
