@@ -57,20 +57,48 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
 
   // ---- bring the candidates on chip in index order: the filter stored them tile by tile, each
   // tile's segment wherever its claim landed; laying the segments out in tile order sorts them.
+  // A warp takes 32 consecutive tiles per step (one per lane for the bookkeeping), then copies
+  // their segments with all lanes, several segments' loads in flight before the first store.
   {
+    const uint32_t warp = tid >> 5;
     uint32_t carry = 0;
     for (uint32_t base = 0; base < n_tiles; base += kSmallThreads) {
       const uint32_t t = base + tid;
       const uint2 sg = t < n_tiles ? seg[(uint64_t)row * n_tiles + t] : make_uint2(0u, 0u);
       uint32_t total;
       const uint32_t dst = carry + block_scan_excl_1024(sg.y, s_warp, &total);
-#pragma unroll 4
-      for (uint32_t i = 0; i < sg.y; ++i) {
-        const uint2 e = c[sg.x + i];
-        s_bits[dst + i] = e.x;
-        s_idx[dst + i] = e.y;
-      }
       carry += total;
+      const uint32_t longest = __reduce_max_sync(0xFFFFFFFFu, sg.y);
+      if (longest == 0u) continue;                 // warp-uniform
+      if (longest <= 32u) {
+        constexpr int kBatch = 8;
+#pragma unroll 1
+        for (int j0 = 0; j0 < 32; j0 += kBatch) {
+          uint2 e[kBatch];
+          uint32_t at[kBatch];
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j) {
+            const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j0 + j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j0 + j);
+            const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j0 + j);
+            at[j] = lane < cnt ? d0 + lane : 0xFFFFFFFFu;
+            if (lane < cnt) e[j] = c[src + lane];
+          }
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j)
+            if (at[j] != 0xFFFFFFFFu) { s_bits[at[j]] = e[j].x; s_idx[at[j]] = e[j].y; }
+        }
+      } else {                                     // some long segment: one tile after the other
+        for (int j = 0; j < 32; ++j) {
+          const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j);
+          const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j);
+          for (uint32_t i = lane; i < cnt; i += 32) {
+            const uint2 e = c[src + i];
+            s_bits[d0 + i] = e.x;
+            s_idx[d0 + i] = e.y;
+          }
+        }
+      }
+      (void)warp;
     }
   }
 
@@ -83,12 +111,23 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     for (int b = tid; b < nbins; b += kSmallThreads) s_hist[b] = 0u;
     __syncthreads();                             // also: the candidate arrays are complete (first pass)
     if (pass == 0) {
-      // the leading digits of the candidates take few distinct values: aggregate equal ones per warp
-      for (uint32_t i = tid; i < n_round; i += kSmallThreads) {
-        const bool on = i < n;
-        const uint32_t digit = on ? ((s_bits[i] & kAbsMask) >> pass_shift(0)) & mask : 0xFFFFFFFFu;
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-        if (on && (peers & lt) == 0u) atomicAdd(&s_hist[digit], (uint32_t)__popc(peers));
+      // Every candidate is >= tau_lo, and most sit within a few leading-digit values of it
+      // (gradient magnitudes fall off fast).  Warp-wide votes and shuffles are scarce on one
+      // SM, so each thread counts the first eight values above tau_lo's in registers over
+      // all its entries; one warp reduction per value at the end.  The rest: plain atomics.
+      const uint32_t d_lo = (rs.tau_lo >> pass_shift(0)) & mask;
+      uint32_t cnt8[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+      for (uint32_t i = tid; i < n; i += kSmallThreads) {
+        const uint32_t digit = ((s_bits[i] & kAbsMask) >> pass_shift(0)) & mask;
+        const uint32_t rel = digit - d_lo;                      // >= 0 for every candidate
+#pragma unroll
+        for (uint32_t b = 0; b < 8; ++b) cnt8[b] += (uint32_t)(rel == b);
+        if (rel >= 8u) atomicAdd(&s_hist[digit], 1u);
+      }
+#pragma unroll
+      for (uint32_t b = 0; b < 8; ++b) {
+        const uint32_t v = __reduce_add_sync(0xFFFFFFFFu, cnt8[b]);
+        if (lane == b && v != 0u) atomicAdd(&s_hist[(d_lo + b) & mask], v);
       }
     } else {
       // later digits are spread out: plain shared-memory atomics of the few entries still in play
@@ -133,39 +172,44 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   }
   const uint32_t tau = prefix, take = k_rem;
 
-  // ---- ordered emission, 1024 candidates per round: an entry is kept if it is above tau, or equal
-  // to tau with fewer than `take` equal entries before it; its output position is the number of
-  // kept entries before it.  Consecutive lanes hold consecutive output positions, so the sign
-  // bits of a warp's kept entries fall into at most two output words (ballot + OR-reduction).
+  // ---- ordered emission, kPer consecutive candidates per thread and round: an entry is kept if
+  // it is above tau, or equal to tau with fewer than `take` equal entries before it; its
+  // output position is the number of kept entries before it.  (Many entries per thread keep
+  // the number of block-wide scans, and with it of warp shuffles, small.)
+  constexpr int kPer = 16;
   uint32_t carry_eq = 0, carry_out = 0;
-  for (uint32_t base = 0; base < n; base += kSmallThreads) {
-    const uint32_t i = base + tid;
-    const bool in = i < n;
-    const uint32_t bits = in ? s_bits[i] : 0u;
-    const uint32_t key = bits & kAbsMask;
-    const bool eq = in && key == tau;
-    uint32_t tot_eq, tot_sel;
-    const uint32_t tie_rank = carry_eq + block_scan_excl_1024(eq ? 1u : 0u, s_warp, &tot_eq);
-    const bool sel = in && (key > tau || (eq && tie_rank < take));
-    const uint32_t pos = carry_out + block_scan_excl_1024(sel ? 1u : 0u, s_warp, &tot_sel);
-    const uint32_t neg = bits >> 31;
-    const bool put = sel && pos < o.K;
-    if (put) {
-      const uint32_t idx = s_idx[i];
-      if (o.idx) o.idx[(uint64_t)row * o.K + pos] = idx;
-      if (o.counter) atomicAdd(o.counter + idx, neg ? -1 : 1);
+  for (uint32_t base = 0; base < n; base += kSmallThreads * kPer) {
+    const uint32_t i0 = base + tid * kPer;
+    uint32_t bits[kPer], eqf = 0, inf = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const bool in = i0 + q < n;
+      bits[q] = in ? s_bits[i0 + q] : 0u;
+      inf |= (uint32_t)in << q;
+      eqf |= (uint32_t)(in && (bits[q] & kAbsMask) == tau) << q;
     }
-    if (o.signbits) {
-      const uint32_t selb = __ballot_sync(0xFFFFFFFFu, put);
-      if (selb) {
-        const uint32_t first = __shfl_sync(0xFFFFFFFFu, pos, __ffs(selb) - 1);   // lowest kept position of the warp
-        const uint32_t w0 = first >> 5;
-        const uint32_t bit = put ? (neg << (pos & 31)) : 0u;
-        const uint32_t v0 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 ? bit : 0u);
-        const uint32_t v1 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 + 1 ? bit : 0u);
-        if (lane == 0) {
-          if (v0) atomicOr(o.signbits + (uint64_t)row * o.words + w0, v0);
-          if (v1) atomicOr(o.signbits + (uint64_t)row * o.words + w0 + 1, v1);
+    uint32_t tot_eq, tot_sel;
+    const uint32_t tie0 = carry_eq + block_scan_excl_1024(__popc(eqf), s_warp, &tot_eq);
+    uint32_t self = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const uint32_t key = bits[q] & kAbsMask;
+      const bool keep = (inf >> q & 1u) &&
+                        (key > tau || ((eqf >> q & 1u) && tie0 + __popc(eqf & ((1u << q) - 1u)) < take));
+      self |= (uint32_t)keep << q;
+    }
+    const uint32_t pos0 = carry_out + block_scan_excl_1024(__popc(self), s_warp, &tot_sel);
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      if (self >> q & 1u) {
+        const uint32_t pos = pos0 + __popc(self & ((1u << q) - 1u));
+        if (pos < o.K) {
+          const uint32_t idx = s_idx[i0 + q];
+          const uint32_t neg = bits[q] >> 31;
+          if (o.idx) o.idx[(uint64_t)row * o.K + pos] = idx;
+          if (o.counter) atomicAdd(o.counter + idx, neg ? -1 : 1);
+          // sign bits only when the message is asked for: one atomic per negative entry
+          if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
         }
       }
     }
