@@ -40,6 +40,13 @@ __device__ __forceinline__ uint32_t block_scan_excl_1024(uint32_t v, uint32_t* s
   return woff + inc - v;
 }
 
+// kOrdered: the message (indices, sign bits) is wanted, so the candidates are laid out in index
+// order and emitted with their output positions.  Otherwise only the votes are wanted, whose
+// order does not matter: the candidates are copied as they lie, every entry above tau votes at
+// once, and only the entries equal to tau are ranked by index among themselves.
+constexpr uint32_t kMaxTiesUnordered = 1024;
+
+template <bool kOrdered>
 __global__ void __launch_bounds__(kSmallThreads, 1)
 select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand, uint32_t cap,
                     const uint2* __restrict__ seg, uint32_t n_tiles, uint32_t* __restrict__ hdr, EmitOut o) {
@@ -55,56 +62,64 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   uint32_t* s_idx = s_bits + n;                               // [n] their indices
   const uint2* c = cand + (uint64_t)row * cap;
 
-  // ---- bring the candidates on chip in index order: the filter stored them tile by tile, each
-  // tile's segment wherever its claim landed; laying the segments out in tile order sorts them.
-  // A warp takes 32 consecutive tiles per step (one per lane for the bookkeeping), then copies
-  // their segments with all lanes, several segments' loads in flight before the first store.
-  {
-    const uint32_t warp = tid >> 5;
-    uint32_t carry = 0;
-    for (uint32_t base = 0; base < n_tiles; base += kSmallThreads) {
-      const uint32_t t = base + tid;
-      const uint2 sg = t < n_tiles ? seg[(uint64_t)row * n_tiles + t] : make_uint2(0u, 0u);
-      uint32_t total;
-      const uint32_t dst = carry + block_scan_excl_1024(sg.y, s_warp, &total);
-      carry += total;
-      const uint32_t longest = __reduce_max_sync(0xFFFFFFFFu, sg.y);
-      if (longest == 0u) continue;                 // warp-uniform
-      if (longest <= 32u) {
-        constexpr int kBatch = 8;
-#pragma unroll 1
-        for (int j0 = 0; j0 < 32; j0 += kBatch) {
-          uint2 e[kBatch];
-          uint32_t at[kBatch];
-#pragma unroll
-          for (int j = 0; j < kBatch; ++j) {
-            const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j0 + j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j0 + j);
-            const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j0 + j);
-            at[j] = lane < cnt ? d0 + lane : 0xFFFFFFFFu;
-            if (lane < cnt) e[j] = c[src + lane];
+  if (!kOrdered) {
+#pragma unroll 8
+    for (uint32_t i = tid; i < n; i += kSmallThreads) {
+      const uint2 e = c[i];
+      s_bits[i] = e.x;
+      s_idx[i] = e.y;
+    }
+  } else {
+    // ---- bring the candidates on chip in index order: the filter stored them tile by tile, each
+    // tile's segment wherever its claim landed; laying the segments out in tile order sorts them.
+    // A warp takes 32 consecutive tiles per step (one per lane for the bookkeeping), then copies
+    // their segments with all lanes, several segments' loads in flight before the first store.
+    {
+      const uint32_t warp = tid >> 5;
+      uint32_t carry = 0;
+      for (uint32_t base = 0; base < n_tiles; base += kSmallThreads) {
+        const uint32_t t = base + tid;
+        const uint2 sg = t < n_tiles ? seg[(uint64_t)row * n_tiles + t] : make_uint2(0u, 0u);
+        uint32_t total;
+        const uint32_t dst = carry + block_scan_excl_1024(sg.y, s_warp, &total);
+        carry += total;
+        const uint32_t longest = __reduce_max_sync(0xFFFFFFFFu, sg.y);
+        if (longest == 0u) continue;                 // warp-uniform
+        if (longest <= 32u) {
+          constexpr int kBatch = 8;
+  #pragma unroll 1
+          for (int j0 = 0; j0 < 32; j0 += kBatch) {
+            uint2 e[kBatch];
+            uint32_t at[kBatch];
+  #pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+              const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j0 + j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j0 + j);
+              const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j0 + j);
+              at[j] = lane < cnt ? d0 + lane : 0xFFFFFFFFu;
+              if (lane < cnt) e[j] = c[src + lane];
+            }
+  #pragma unroll
+            for (int j = 0; j < kBatch; ++j)
+              if (at[j] != 0xFFFFFFFFu) { s_bits[at[j]] = e[j].x; s_idx[at[j]] = e[j].y; }
           }
-#pragma unroll
-          for (int j = 0; j < kBatch; ++j)
-            if (at[j] != 0xFFFFFFFFu) { s_bits[at[j]] = e[j].x; s_idx[at[j]] = e[j].y; }
-        }
-      } else {                                     // some long segment: one tile after the other
-        for (int j = 0; j < 32; ++j) {
-          const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j);
-          const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j);
-          for (uint32_t i = lane; i < cnt; i += 32) {
-            const uint2 e = c[src + i];
-            s_bits[d0 + i] = e.x;
-            s_idx[d0 + i] = e.y;
+        } else {                                     // some long segment: one tile after the other
+          for (int j = 0; j < 32; ++j) {
+            const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j);
+            const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j);
+            for (uint32_t i = lane; i < cnt; i += 32) {
+              const uint2 e = c[src + i];
+              s_bits[d0 + i] = e.x;
+              s_idx[d0 + i] = e.y;
+            }
           }
         }
+        (void)warp;
       }
-      (void)warp;
     }
   }
 
   // ---- radix select: tau = K-th largest magnitude, take = how many entries equal to tau are kept
-  uint32_t prefix = 0, k_rem = o.K;
-  const uint32_t n_round = (n + 31u) & ~31u;
+  uint32_t prefix = 0, k_rem = o.K, n_equal = 0;
   for (int pass = 0; pass < kNumPasses; ++pass) {
     const int nbins = 1 << pass_bits(pass);
     const uint32_t mask = (uint32_t)(nbins - 1);
@@ -162,6 +177,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     }
     __syncthreads();
     uint32_t digit = s_sel[0], a = s_sel[1];
+    n_equal = digit == 0xFFFFFFFFu ? 0u : s_hist[digit];        // after the last pass: entries equal to tau
     if (digit == 0xFFFFFFFFu) {                          // fewer than k_rem entries: cannot happen for a valid row
       if (tid == 0) atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
       digit = 0u; a = 0u;
@@ -171,6 +187,52 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     __syncthreads();                             // s_sel and s_hist are reused by the next pass
   }
   const uint32_t tau = prefix, take = k_rem;
+
+  if (!kOrdered) {
+    // ---- votes only.  Entries equal to tau are few as a rule; they are kept by ascending index
+    // until `take` are taken, which needs their rank among themselves only.
+    const bool rank_ties = n_equal > take;                       // otherwise every one of them is kept
+    if (rank_ties && n_equal > kMaxTiesUnordered) return;        // too many to rank here: the general passes do this row
+    uint32_t* s_tie_idx = s_hist;                                // the histogram is no longer needed
+    uint32_t* s_tie_neg = s_hist + kMaxTiesUnordered;
+    if (tid == 0) s_sel[0] = 0u;
+    __syncthreads();
+#pragma unroll 4
+    for (uint32_t i = tid; i < n; i += kSmallThreads) {
+      const uint32_t bits = s_bits[i], key = bits & kAbsMask;
+      if (key > tau || (key == tau && !rank_ties)) {
+        atomicAdd(o.counter + s_idx[i], (bits >> 31) ? -1 : 1);
+      } else if (key == tau) {
+        const uint32_t slot = atomicAdd(&s_sel[0], 1u);
+        s_tie_idx[slot] = s_idx[i];
+        s_tie_neg[slot] = bits >> 31;
+      }
+    }
+    uint32_t n_kept = o.K;
+    if (rank_ties) {
+      __syncthreads();
+      const uint32_t e = s_sel[0];                               // == n_equal
+      if (tid < e) {
+        const uint32_t mine = s_tie_idx[tid];
+        uint32_t before = 0;
+        for (uint32_t j = 0; j < e; ++j) before += (uint32_t)(s_tie_idx[j] < mine);
+        if (before < take) atomicAdd(o.counter + mine, s_tie_neg[tid] ? -1 : 1);
+      }
+      if (e != n_equal) n_kept = 0xFFFFFFFFu;                    // cannot happen
+    }
+    if (tid == 0) {
+      rows[row].tau = tau;
+      rows[row].take_ties = take;
+      rows[row].n_emitted = n_kept;
+      rows[row].done = 1u;
+      if (n_kept != o.K) {
+        atomicAdd(hdr + kHdrBadCount, 1u);
+        atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
+      }
+      atomicMax(hdr + kHdrMaxCand, n);
+    }
+    return;
+  }
 
   // ---- ordered emission, kPer consecutive candidates per thread and round: an entry is kept if
   // it is above tau, or equal to tau with fewer than `take` equal entries before it; its
@@ -236,10 +298,11 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
   // enough dynamic shared memory for the largest row this kernel accepts
   uint64_t need = (uint64_t)L.cap * 8u;
   if (need > kSmallSelectBytes) need = kSmallSelectBytes;
-  cudaError_t e = cudaFuncSetAttribute(select_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)kSmallSelectBytes);
+  const bool ordered = o.idx != nullptr || o.signbits != nullptr || o.counter == nullptr;
+  auto kernel = ordered ? select_small_kernel<true> : select_small_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
   if (e != cudaSuccess) return e;
-  select_small_kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, cand, L.cap, seg, L.n_tiles, hdr, o);
+  kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, cand, L.cap, seg, L.n_tiles, hdr, o);
   e = cudaGetLastError();
   if (e == cudaSuccess) count_launch();
   return e;
