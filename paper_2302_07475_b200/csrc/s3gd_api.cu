@@ -21,7 +21,7 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   if (M <= 0 || M > 65535 || d == 0 || d >= (1ull << 32) || K > d) return false;
   L->M = M; L->d = d; L->K = K;
   L->n_tiles = (uint32_t)((d + kTileElems - 1) / kTileElems);
-  L->cap = 0; L->n_sample = 0; L->j_rank = 0; L->sample_stride = 0;
+  L->cap = 0; L->typical_cand = 0; L->n_sample = 0; L->j_rank = 0; L->sample_stride = 0;
   const bool use_filter = K > 0 && K < d && K * 4 <= d;
   if (use_filter) {
     const double p = (double)K / (double)d;
@@ -46,6 +46,9 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
     if (cap < (double)K) cap = (double)K;
     if (cap > (double)d) cap = (double)d;
     L->cap = (uint32_t)cap;
+    double typical = ceil(r * j * 1.25);
+    if (typical > cap) typical = cap;
+    L->typical_cand = (uint32_t)typical;
   }
   size_t off = 0;
   L->off_hdr = off;      off = align_up(off + kHdrWords * sizeof(uint32_t), 256);

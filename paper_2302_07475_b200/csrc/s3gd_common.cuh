@@ -61,6 +61,7 @@ struct Layout {
   int M;
   uint32_t n_tiles;      // tiles per row
   uint32_t cap;          // candidate capacity per row
+  uint32_t typical_cand; // survivors a row is expected to have (mean of the sampling plan plus grid slack)
   uint32_t n_sample;     // sampled entries per row
   uint32_t j_rank;       // sample rank that fixes tau_lo
   uint32_t sample_stride;  // distance between sampled groups of 8 (0: whole row sampled)

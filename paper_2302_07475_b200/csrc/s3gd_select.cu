@@ -51,17 +51,13 @@ __device__ __forceinline__ bool last_block_of_row(uint32_t* ticket, uint32_t n_b
 }
 
 // ------------------------------------------------------- histogram passes
-// Shared-memory histogram.  In the first pass the leading digits take few distinct values
-// (gradient exponents cluster), so increments are warp-aggregated: lanes that hit the same
-// bin elect a leader which adds their count once.  In the later passes only the entries of
-// one first-pass bin are still in play and their digits are spread out: plain atomics.
-__device__ __forceinline__ void hist_add(uint32_t* s_hist, bool on, uint32_t digit, bool aggregate) {
-  if (aggregate) {
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? digit : 0xFFFFFFFFu);
-    if (on && (peers & lanemask_lt()) == 0u) atomicAdd(&s_hist[digit], (uint32_t)__popc(peers));
-  } else if (on) {
-    atomicAdd(&s_hist[digit], 1u);
-  }
+// Shared-memory histogram with warp-aggregated increments: lanes that hit the same
+// bin elect a leader which adds their count once (gradient magnitudes cluster in a
+// few bins, and quantised gradients do so in every pass, so plain atomics would
+// serialise on those bins).
+__device__ __forceinline__ void hist_add(uint32_t* s_hist, bool on, uint32_t digit) {
+  const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? digit : 0xFFFFFFFFu);
+  if (on && (peers & lanemask_lt()) == 0u) atomicAdd(&s_hist[digit], (uint32_t)__popc(peers));
 }
 
 __device__ __forceinline__ bool in_prefix(uint32_t key, uint32_t prefix, int pass) {
@@ -143,7 +139,7 @@ __global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* 
       bool on = i < n;
       const uint32_t key = on ? (c[i].x & kAbsMask) : 0u;
       on = on && in_prefix(key, rs.prefix, pass);
-      hist_add(s_hist, on, (key >> pass_shift(pass)) & mask, pass == 0);
+      hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
     }
   } else if (!is_c && !use_c) {
     worked = true;
@@ -157,7 +153,7 @@ __global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* 
       load_tile(T, rowp, d, head, t);
       if (t == 0 && threadIdx.x < 32) {
         const uint32_t key = T.head_bits & kAbsMask;
-        hist_add(s_hist, T.head_valid && in_prefix(key, rs.prefix, pass), (key >> pass_shift(pass)) & mask, pass == 0);
+        hist_add(s_hist, T.head_valid && in_prefix(key, rs.prefix, pass), (key >> pass_shift(pass)) & mask);
       }
 #pragma unroll
       for (int it = 0; it < kTileIters; ++it) {
@@ -165,7 +161,7 @@ __global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* 
         for (int q = 0; q < 4; ++q) {
           const uint32_t key = T.bits[it][q] & kAbsMask;
           const bool on = (T.valid[it] >> q & 1u) && in_prefix(key, rs.prefix, pass);
-          hist_add(s_hist, on, (key >> pass_shift(pass)) & mask, pass == 0);
+          hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
         }
       }
     }

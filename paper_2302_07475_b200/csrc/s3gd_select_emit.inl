@@ -337,11 +337,13 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     cudaError_t e = launch_select_small(L, rows, cand, seg, hdr, o, st);
     if (e != cudaSuccess) return e;
   }
-  // Blocks per row (each block strides over its row's candidates or tiles): about four CTAs
-  // per SM over all rows, never more than the work can use.  Rows finished by the single-CTA
-  // selection cost these launches only an early exit.
-  const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * 4 + M - 1) / M);
-  const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, per_row) : 0u;
+  // Blocks per row (each block strides over its row's candidates or tiles).  If a row's
+  // candidates are expected to fit the single-CTA selection, these launches only serve the
+  // odd row that did not fit or fell back to the whole-row route, and normally exit at once:
+  // keep them small.  Otherwise they carry the selection of all rows: about eight CTAs per SM.
+  const bool only_fallback = use_filter && fits_single_cta(L.typical_cand);
+  const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * (only_fallback ? 4 : 8) + M - 1) / M);
+  const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
   for (int pass = 0; pass < kNumPasses; ++pass) {
