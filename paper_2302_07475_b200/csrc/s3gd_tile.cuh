@@ -74,7 +74,8 @@ __device__ __forceinline__ void load_tile(Tile& T, const uint32_t* __restrict__ 
 // Ranks of flagged entries in ascending-index order.
 // flags[it] (low 4 bits) and head_flag mark entries; after the call
 //   rank of (it, slot) = lane_excl(it) + popc(flags[it] & ((1u << slot) - 1))  + block offset of (warp, it)
-// which rank_of() evaluates.  Uses s_wtot[kWarpsPerTile + 1] shared words and two barriers.
+// which rank_of() evaluates.  Uses s_wtot[kWarpsPerTile + 1] shared words; tile_ranks() is the
+// two-barrier form, tile_ranks_publish()/tile_ranks_collect() let the caller own the barrier.
 struct TileRanks {
   uint32_t lane_excl[kTileIters];  // flagged entries of this warp-iteration in lower lanes
   uint32_t it_off[kTileIters];     // flagged entries of this warp in earlier iterations
@@ -83,8 +84,10 @@ struct TileRanks {
   uint32_t tile_total;             // all flagged entries of the tile
 };
 
-__device__ __forceinline__ void tile_ranks(TileRanks& R, const uint32_t (&flags)[kTileIters], bool head_flag,
-                                           uint32_t* s_wtot) {
+// First half: per-warp packed scan; publishes this warp's total (and the head count) in
+// s_wtot[0..kWarpsPerTile].  The caller places one block barrier between the halves.
+__device__ __forceinline__ void tile_ranks_publish(TileRanks& R, const uint32_t (&flags)[kTileIters], bool head_flag,
+                                                   uint32_t* s_wtot) {
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // counts are <= 4 per lane and <= 128 per warp-iteration, so the counts of four
   // iterations travel through the scan as the 8-bit fields of one word
@@ -94,46 +97,62 @@ __device__ __forceinline__ void tile_ranks(TileRanks& R, const uint32_t (&flags)
     lo |= (uint32_t)__popc(flags[it] & 0xFu) << (8 * it);
     hi |= (uint32_t)__popc(flags[it + 4] & 0xFu) << (8 * it);
   }
-  uint32_t ilo = lo, ihi = hi;      // inclusive scans over lanes
-#pragma unroll
-  for (int s = 1; s < 32; s <<= 1) {
-    uint32_t a = __shfl_up_sync(0xFFFFFFFFu, ilo, s);
-    uint32_t b = __shfl_up_sync(0xFFFFFFFFu, ihi, s);
-    if (lane >= (uint32_t)s) { ilo += a; ihi += b; }
-  }
-  // a full warp-iteration holds 128 flagged entries: 128 fits the 8-bit field (max 255)
-  const uint32_t tlo = __shfl_sync(0xFFFFFFFFu, ilo, 31), thi = __shfl_sync(0xFFFFFFFFu, ihi, 31);
-  const uint32_t elo = ilo - lo, ehi = ihi - hi;
   uint32_t run = 0;
+  if (__any_sync(0xFFFFFFFFu, (lo | hi) != 0u)) {
+    uint32_t ilo = lo, ihi = hi;      // inclusive scans over lanes
 #pragma unroll
-  for (int it = 0; it < 4; ++it) {
-    R.lane_excl[it] = (elo >> (8 * it)) & 0xFFu;
-    R.it_off[it] = run;
-    run += (tlo >> (8 * it)) & 0xFFu;
-  }
+    for (int s = 1; s < 32; s <<= 1) {
+      uint32_t a = __shfl_up_sync(0xFFFFFFFFu, ilo, s);
+      uint32_t b = __shfl_up_sync(0xFFFFFFFFu, ihi, s);
+      if (lane >= (uint32_t)s) { ilo += a; ihi += b; }
+    }
+    // a full warp-iteration holds 128 flagged entries: 128 fits the 8-bit field (max 255)
+    const uint32_t tlo = __shfl_sync(0xFFFFFFFFu, ilo, 31), thi = __shfl_sync(0xFFFFFFFFu, ihi, 31);
+    const uint32_t elo = ilo - lo, ehi = ihi - hi;
 #pragma unroll
-  for (int it = 0; it < 4; ++it) {
-    R.lane_excl[it + 4] = (ehi >> (8 * it)) & 0xFFu;
-    R.it_off[it + 4] = run;
-    run += (thi >> (8 * it)) & 0xFFu;
+    for (int it = 0; it < 4; ++it) {
+      R.lane_excl[it] = (elo >> (8 * it)) & 0xFFu;
+      R.it_off[it] = run;
+      run += (tlo >> (8 * it)) & 0xFFu;
+    }
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      R.lane_excl[it + 4] = (ehi >> (8 * it)) & 0xFFu;
+      R.it_off[it + 4] = run;
+      run += (thi >> (8 * it)) & 0xFFu;
+    }
+  } else {                                         // nothing flagged in this warp: no scan needed
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it) { R.lane_excl[it] = 0u; R.it_off[it] = 0u; }
   }
   const uint32_t hb = __ballot_sync(0xFFFFFFFFu, head_flag);   // only warp 0 can have head entries
   R.head_rank = __popc(hb & lanemask_lt());
-  __syncthreads();                       // previous users of s_wtot are done
   if (lane == 0) {
     s_wtot[warp] = run;
     if (warp == 0) s_wtot[kWarpsPerTile] = __popc(hb);
   }
-  __syncthreads();
+}
+
+// Second half (after the barrier): offsets of this warp and the tile total.
+__device__ __forceinline__ void tile_ranks_collect(TileRanks& R, const uint32_t* s_wtot) {
+  const uint32_t warp = threadIdx.x >> 5;
   uint32_t off = s_wtot[kWarpsPerTile], tot = off;
 #pragma unroll
   for (int w = 0; w < kWarpsPerTile; ++w) {
-    uint32_t c = s_wtot[w];
+    const uint32_t c = s_wtot[w];
     if ((uint32_t)w < warp) off += c;
     tot += c;
   }
   R.warp_off = off;
   R.tile_total = tot;
+}
+
+__device__ __forceinline__ void tile_ranks(TileRanks& R, const uint32_t (&flags)[kTileIters], bool head_flag,
+                                           uint32_t* s_wtot) {
+  __syncthreads();                       // previous users of s_wtot are done
+  tile_ranks_publish(R, flags, head_flag, s_wtot);
+  __syncthreads();
+  tile_ranks_collect(R, s_wtot);
 }
 
 __device__ __forceinline__ uint32_t rank_of(const TileRanks& R, const uint32_t (&flags)[kTileIters], int it, int slot) {

@@ -254,6 +254,29 @@ def test_rows_that_leave_the_single_read_route():
     assert info[1] == M - 1
 
 
+@pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900)])
+def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
+    """Many entries exactly at the K-th magnitude, more than are taken: the lowest indices must win.
+
+    Sized so that the row's survivors fit the single-CTA selection; 600 ties are ranked there,
+    3000 are more than it ranks on chip and the row goes to the general passes instead.
+    """
+    M, d, n_big = 3, 200_000, 1000
+    g = torch.Generator("cpu").manual_seed(n_ties * 7 + take)
+    rows = []
+    for m in range(M):
+        v = (torch.rand(d, generator=g) * 0.9).float()                       # below 1: never selected
+        perm = torch.randperm(d, generator=g)
+        v[perm[:n_big]] = 5.0 + torch.rand(n_big, generator=g)               # clearly above the threshold
+        v[perm[n_big:n_big + n_ties]] = 2.0                                  # the ties
+        sign = torch.where(torch.rand(d, generator=g) < 0.5, -1.0, 1.0)
+        rows.append(v * sign)
+    grads = torch.stack(rows).contiguous().to(DEV)
+    x = torch.zeros(d, device=DEV)
+    info = check_all(grads, x, n_big + take, 0.25, tag=f"ties {n_ties}/{take}")
+    assert info[1] == 0                      # no row fell back to the whole-row route
+
+
 def test_majority_vote_semantics_and_range_flag():
     d, M, K = 10, 2, 4
     idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)
