@@ -120,90 +120,137 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   if (lane == 0) rows[row].tau_lo = result << 16;
 }
 
-// Persistent CTAs over (row, tile).  Survivors of a tile are appended to the row's
-// candidate list in ascending index order; the list position of a tile is claimed
-// with one atomic, and (position, count) is recorded per tile so that later passes
-// can walk a row's candidates in index order without sorting.
+// Persistent CTAs over (row, tile); CTA c takes the items c, c + gridDim.x, ...  Survivors of a
+// tile are appended to the row's candidate list in ascending index order; the list position
+// of a tile is claimed with one atomic, and (position, count) is recorded per tile so that
+// later passes can walk a row's candidates in index order without sorting.
 //
-// One block barrier per tile and no wait on the claim: the survivors of tile k are
-// first staged in shared memory at their rank; the atomic that claims their list
-// position is issued and left in flight; after the barrier of tile k+1 -- a whole
-// tile of loads and compares later -- its result is there and the staged survivors
-// are copied out, coalesced.  Tiles with more survivors than the staging buffer holds
-// (dense regions) claim and store directly, with one more barrier.
-constexpr int kStageCap = 512;                 // survivors staged per tile (8 bytes each, two buffers)
+// Fast path (whole tile inside the row, no warp with more than kWarpStage survivors): a warp
+// tests its 1024 entries 128 at a time; only iterations in which some lane has a survivor (a
+// warp vote) are ranked, by ballot, and their survivors go to the warp's staging list in
+// shared memory.  One block barrier per tile publishes the eight warp counts.  The atomic
+// that claims the list position is issued and left in flight; after the barrier of the NEXT
+// tile -- a whole tile of loads and compares later -- its result is there and every warp
+// copies its staged survivors out.
+// Other tiles (the ragged last tile of a row, dense regions) are ranked in registers with a
+// packed scan, claim at once and store directly, with more barriers.
+constexpr int kWarpStage = 64;                 // survivors a warp can stage per tile (8 bytes each, two buffers)
 
 // magnitude >= tau_lo, decided on the float value: |x| < tau is false for NaN, whose bit
 // pattern is above every threshold, so !(|x| < tau) agrees with the unsigned compare of the
 // sign-less bit patterns for every input (denormals are not flushed in this build).
-__device__ __forceinline__ uint32_t hit(uint32_t b, float tau) { return (uint32_t)!(fabsf(__uint_as_float(b)) < tau); }
+__device__ __forceinline__ bool hit(uint32_t b, float tau) { return !(fabsf(__uint_as_float(b)) < tau); }
 
 __global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
-                                                              RowState* __restrict__ rows, uint2* __restrict__ cand,
-                                                              uint32_t cap, uint2* __restrict__ seg,
-                                                              uint32_t n_tiles) {
-  __shared__ uint2 s_stage[2][kStageCap];
-  __shared__ uint32_t s_wtot[2][kWarpsPerTile + 1];
+                                                                 RowState* __restrict__ rows,
+                                                                 uint2* __restrict__ cand, uint32_t cap,
+                                                                 uint2* __restrict__ seg, uint32_t n_tiles) {
+  __shared__ uint2 s_stage[2][kWarpsPerTile][kWarpStage];
+  __shared__ __align__(16) uint32_t s_wtot[3][kWarpsPerTile];   // survivors per warp of tile k in slot k % 3
   __shared__ uint32_t s_base[2];
-  __shared__ uint32_t s_direct_base;
-  const uint32_t tid = threadIdx.x, lane = tid & 31;
+  __shared__ uint32_t s_slow_wtot[kWarpsPerTile + 1];
+  __shared__ uint32_t s_slow_base;
+  const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, lt = lanemask_lt();
   const uint64_t n_work = (uint64_t)M * n_tiles;
+  if (blockIdx.x >= n_work) return;
+  // walk (row, tile) without dividing in the loop
+  uint32_t row = (uint32_t)(blockIdx.x / n_tiles), t = (uint32_t)(blockIdx.x - (uint64_t)row * n_tiles);
+  uint32_t cur_row = 0xFFFFFFFFu, head = 0;
+  const uint32_t* rowp = gbits;
+  float tau = 0.f;
   uint32_t pend_n = 0, pend_row = 0, pend_t = 0;   // staged survivors of the previous tile (uniform)
   uint32_t pend_base = 0;                          // thread 0: the claim made for them (may still be in flight)
-  int par = 0;
-  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x, par ^= 1) {
-    const uint32_t row = (uint32_t)(w / n_tiles), t = (uint32_t)(w - (uint64_t)row * n_tiles);
-    const uint32_t* rowp = gbits + (uint64_t)row * d;
-    const uint32_t head = row_head(rowp, d);
-    const float tau = __uint_as_float(rows[row].tau_lo);
+  uint32_t k = 0;
+  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x, ++k) {
+    if (row != cur_row) {
+      cur_row = row;
+      rowp = gbits + (uint64_t)row * d;
+      head = row_head(rowp, d);
+      tau = __uint_as_float(rows[row].tau_lo);
+    }
+    const int par = (int)(k & 1), slot = (int)(k % 3), prev_slot = (slot + 2) % 3;
+    const bool whole = (uint64_t)head + (uint64_t)(t + 1) * kTileElems <= d;
     Tile T;
     load_tile(T, rowp, d, head, t);
-    uint32_t flags[kTileIters];
+    uint32_t run = 0;                              // survivors of this warp so far (uniform in the warp)
+    if (whole) {
+      uint2* wl = s_stage[par][warp];
+      if (T.head_valid || (t == 0 && head != 0u && warp == 0)) {      // warp 0 of a row's first tile
+        const uint32_t hb = __ballot_sync(0xFFFFFFFFu, T.head_valid && hit(T.head_bits, tau));
+        if (hb >> lane & 1u) wl[__popc(hb & lt)] = make_uint2(T.head_bits, lane);
+        run = __popc(hb);
+      }
+      const uint32_t idx0 = (uint32_t)T.e0;
 #pragma unroll
-    for (int it = 0; it < kTileIters; ++it)
-      flags[it] = (hit(T.bits[it][0], tau) | (hit(T.bits[it][1], tau) << 1) | (hit(T.bits[it][2], tau) << 2) |
-                   (hit(T.bits[it][3], tau) << 3)) & T.valid[it];
-    const bool head_flag = T.head_valid && hit(T.head_bits, tau);
-    TileRanks R;
-    tile_ranks_publish(R, flags, head_flag, s_wtot[par]);
+      for (int it = 0; it < kTileIters; ++it) {
+        const bool h0 = hit(T.bits[it][0], tau), h1 = hit(T.bits[it][1], tau);
+        const bool h2 = hit(T.bits[it][2], tau), h3 = hit(T.bits[it][3], tau);
+        if (__any_sync(0xFFFFFFFFu, h0 | h1 | h2 | h3)) {
+          const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, h0), b1 = __ballot_sync(0xFFFFFFFFu, h1);
+          const uint32_t b2 = __ballot_sync(0xFFFFFFFFu, h2), b3 = __ballot_sync(0xFFFFFFFFu, h3);
+          uint32_t pos = run + __popc(b0 & lt) + __popc(b1 & lt) + __popc(b2 & lt) + __popc(b3 & lt);
+          const uint32_t idx = idx0 + it * 128;
+          if (h0) { if (pos < (uint32_t)kWarpStage) wl[pos] = make_uint2(T.bits[it][0], idx); ++pos; }
+          if (h1) { if (pos < (uint32_t)kWarpStage) wl[pos] = make_uint2(T.bits[it][1], idx + 1); ++pos; }
+          if (h2) { if (pos < (uint32_t)kWarpStage) wl[pos] = make_uint2(T.bits[it][2], idx + 2); ++pos; }
+          if (h3) { if (pos < (uint32_t)kWarpStage) wl[pos] = make_uint2(T.bits[it][3], idx + 3); }
+          run += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
+        }
+      }
+    }
+    if (lane == 0) s_wtot[slot][warp] = run;       // may exceed kWarpStage: the tile then takes the other path
     if (tid == 0 && pend_n) {                      // the claim of the previous tile has had a tile's time to return
       s_base[par ^ 1] = pend_base;
       seg[(uint64_t)pend_row * n_tiles + pend_t] = make_uint2(pend_base, pend_n);
     }
     __syncthreads();
-    if (pend_n) {                                  // copy out the previous tile's survivors
-      const uint32_t base = s_base[par ^ 1];
-      uint2* out = cand + (uint64_t)pend_row * cap;
-      for (uint32_t i = tid; i < pend_n; i += kTileThreads)
-        if (base + i < cap) out[base + i] = s_stage[par ^ 1][i];
-    }
-    tile_ranks_collect(R, s_wtot[par]);
-    const uint32_t total = R.tile_total;
-    if (total == 0u) {
-      if (tid == 0) seg[(uint64_t)row * n_tiles + t] = make_uint2(0u, 0u);
-      pend_n = 0;
-      continue;
-    }
-    if (total <= (uint32_t)kStageCap) {
-      if (head_flag) s_stage[par][R.head_rank] = make_uint2(T.head_bits, lane);
+    if (pend_n) {                                  // every warp copies out what it staged for the previous tile
+      const uint4 a = *reinterpret_cast<const uint4*>(&s_wtot[prev_slot][0]);
+      const uint4 b = *reinterpret_cast<const uint4*>(&s_wtot[prev_slot][4]);
+      const uint32_t c[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+      uint32_t off = s_base[par ^ 1], n = 0;
 #pragma unroll
-      for (int it = 0; it < kTileIters; ++it) {
-        if (flags[it] == 0u) continue;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          if (flags[it] >> q & 1u)
-            s_stage[par][rank_of(R, flags, it, q)] = make_uint2(T.bits[it][q], (uint32_t)(T.first(it) + q));
+      for (int wv = 0; wv < kWarpsPerTile; ++wv) {
+        off += (uint32_t)wv < warp ? c[wv] : 0u;
+        n = (uint32_t)wv == warp ? c[wv] : n;
       }
-      if (tid == 0) pend_base = atomicAdd(&rows[row].n_cand, total);
-      pend_n = total; pend_row = row; pend_t = t;
-    } else {                                       // dense tile: claim now, store from registers
+      uint2* out = cand + (uint64_t)pend_row * cap;
+      for (uint32_t i = lane; i < n; i += 32)
+        if (off + i < cap) out[off + i] = s_stage[par ^ 1][warp][i];
+    }
+    uint32_t total, wmax;
+    {
+      const uint4 a = *reinterpret_cast<const uint4*>(&s_wtot[slot][0]);
+      const uint4 b = *reinterpret_cast<const uint4*>(&s_wtot[slot][4]);
+      total = a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w;
+      wmax = max(max(max(a.x, a.y), max(a.z, a.w)), max(max(b.x, b.y), max(b.z, b.w)));
+    }
+    if (whole && wmax <= (uint32_t)kWarpStage) {
+      if (total != 0u) {
+        if (tid == 0) pend_base = atomicAdd(&rows[row].n_cand, total);
+        pend_row = row; pend_t = t;
+      } else if (tid == 0) {
+        seg[(uint64_t)row * n_tiles + t] = make_uint2(0u, 0u);
+      }
+      pend_n = total;
+    } else {
+      // ragged or dense tile: flags and ranks in registers, claim now, store directly
+      pend_n = 0;
+      uint32_t flags[kTileIters];
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it)
+        flags[it] = ((uint32_t)hit(T.bits[it][0], tau) | ((uint32_t)hit(T.bits[it][1], tau) << 1) |
+                     ((uint32_t)hit(T.bits[it][2], tau) << 2) | ((uint32_t)hit(T.bits[it][3], tau) << 3)) & T.valid[it];
+      const bool head_flag = T.head_valid && hit(T.head_bits, tau);
+      TileRanks R;
+      tile_ranks(R, flags, head_flag, s_slow_wtot);
       if (tid == 0) {
-        const uint32_t b = atomicAdd(&rows[row].n_cand, total);
-        s_direct_base = b;
-        seg[(uint64_t)row * n_tiles + t] = make_uint2(b, total);
+        const uint32_t bse = R.tile_total ? atomicAdd(&rows[row].n_cand, R.tile_total) : 0u;
+        s_slow_base = bse;
+        seg[(uint64_t)row * n_tiles + t] = make_uint2(bse, R.tile_total);
       }
       __syncthreads();
-      const uint32_t base = s_direct_base;
+      const uint32_t base = s_slow_base;
       uint2* out = cand + (uint64_t)row * cap;
       if (head_flag && base + R.head_rank < cap) out[base + R.head_rank] = make_uint2(T.head_bits, lane);
 #pragma unroll
@@ -217,19 +264,28 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t*
           }
         }
       }
-      pend_n = 0;
     }
+    // next item of this CTA
+    uint64_t nt = (uint64_t)t + gridDim.x;
+    while (nt >= n_tiles) { nt -= n_tiles; ++row; }
+    t = (uint32_t)nt;
   }
   if (pend_n) {                                    // the last tile's survivors
+    const int par = (int)((k - 1) & 1), slot = (int)((k - 1) % 3);
     if (tid == 0) {
-      s_base[par ^ 1] = pend_base;
+      s_base[par] = pend_base;
       seg[(uint64_t)pend_row * n_tiles + pend_t] = make_uint2(pend_base, pend_n);
     }
     __syncthreads();
-    const uint32_t base = s_base[par ^ 1];
+    uint32_t off = s_base[par], n = 0;
+#pragma unroll
+    for (int wv = 0; wv < kWarpsPerTile; ++wv) {
+      off += (uint32_t)wv < warp ? s_wtot[slot][wv] : 0u;
+      n = (uint32_t)wv == warp ? s_wtot[slot][wv] : n;
+    }
     uint2* out = cand + (uint64_t)pend_row * cap;
-    for (uint32_t i = tid; i < pend_n; i += kTileThreads)
-      if (base + i < cap) out[base + i] = s_stage[par ^ 1][i];
+    for (uint32_t i = lane; i < n; i += 32)
+      if (off + i < cap) out[off + i] = s_stage[par][warp][i];
   }
 }
 
