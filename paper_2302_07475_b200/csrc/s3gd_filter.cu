@@ -289,6 +289,106 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t*
   }
 }
 
+// ---- the same pass for denser survivors (more than about one in 250 entries): nearly every
+// 128-entry iteration then holds a survivor, so ranking all of them with one packed warp scan
+// is cheaper than a vote and four ballots per iteration; survivors are staged per CTA.
+constexpr int kStageCap = 512;                 // survivors staged per tile (8 bytes each, two buffers)
+
+__global__ void __launch_bounds__(kTileThreads, 4) filter_scan_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
+                                                              RowState* __restrict__ rows, uint2* __restrict__ cand,
+                                                              uint32_t cap, uint2* __restrict__ seg,
+                                                              uint32_t n_tiles) {
+  __shared__ uint2 s_stage[2][kStageCap];
+  __shared__ uint32_t s_wtot[2][kWarpsPerTile + 1];
+  __shared__ uint32_t s_base[2];
+  __shared__ uint32_t s_direct_base;
+  const uint32_t tid = threadIdx.x, lane = tid & 31;
+  const uint64_t n_work = (uint64_t)M * n_tiles;
+  uint32_t pend_n = 0, pend_row = 0, pend_t = 0;   // staged survivors of the previous tile (uniform)
+  uint32_t pend_base = 0;                          // thread 0: the claim made for them (may still be in flight)
+  int par = 0;
+  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x, par ^= 1) {
+    const uint32_t row = (uint32_t)(w / n_tiles), t = (uint32_t)(w - (uint64_t)row * n_tiles);
+    const uint32_t* rowp = gbits + (uint64_t)row * d;
+    const uint32_t head = row_head(rowp, d);
+    const float tau = __uint_as_float(rows[row].tau_lo);
+    Tile T;
+    load_tile(T, rowp, d, head, t);
+    uint32_t flags[kTileIters];
+#pragma unroll
+    for (int it = 0; it < kTileIters; ++it)
+      flags[it] = ((uint32_t)hit(T.bits[it][0], tau) | ((uint32_t)hit(T.bits[it][1], tau) << 1) |
+                   ((uint32_t)hit(T.bits[it][2], tau) << 2) | ((uint32_t)hit(T.bits[it][3], tau) << 3)) & T.valid[it];
+    const bool head_flag = T.head_valid && hit(T.head_bits, tau);
+    TileRanks R;
+    tile_ranks_publish(R, flags, head_flag, s_wtot[par]);
+    if (tid == 0 && pend_n) {                      // the claim of the previous tile has had a tile's time to return
+      s_base[par ^ 1] = pend_base;
+      seg[(uint64_t)pend_row * n_tiles + pend_t] = make_uint2(pend_base, pend_n);
+    }
+    __syncthreads();
+    if (pend_n) {                                  // copy out the previous tile's survivors
+      const uint32_t base = s_base[par ^ 1];
+      uint2* out = cand + (uint64_t)pend_row * cap;
+      for (uint32_t i = tid; i < pend_n; i += kTileThreads)
+        if (base + i < cap) out[base + i] = s_stage[par ^ 1][i];
+    }
+    tile_ranks_collect(R, s_wtot[par]);
+    const uint32_t total = R.tile_total;
+    if (total == 0u) {
+      if (tid == 0) seg[(uint64_t)row * n_tiles + t] = make_uint2(0u, 0u);
+      pend_n = 0;
+      continue;
+    }
+    if (total <= (uint32_t)kStageCap) {
+      if (head_flag) s_stage[par][R.head_rank] = make_uint2(T.head_bits, lane);
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it) {
+        if (flags[it] == 0u) continue;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (flags[it] >> q & 1u)
+            s_stage[par][rank_of(R, flags, it, q)] = make_uint2(T.bits[it][q], (uint32_t)(T.first(it) + q));
+      }
+      if (tid == 0) pend_base = atomicAdd(&rows[row].n_cand, total);
+      pend_n = total; pend_row = row; pend_t = t;
+    } else {                                       // dense tile: claim now, store from registers
+      if (tid == 0) {
+        const uint32_t b = atomicAdd(&rows[row].n_cand, total);
+        s_direct_base = b;
+        seg[(uint64_t)row * n_tiles + t] = make_uint2(b, total);
+      }
+      __syncthreads();
+      const uint32_t base = s_direct_base;
+      uint2* out = cand + (uint64_t)row * cap;
+      if (head_flag && base + R.head_rank < cap) out[base + R.head_rank] = make_uint2(T.head_bits, lane);
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it) {
+        if (flags[it] == 0u) continue;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (flags[it] >> q & 1u) {
+            const uint32_t pos = base + rank_of(R, flags, it, q);
+            if (pos < cap) out[pos] = make_uint2(T.bits[it][q], (uint32_t)(T.first(it) + q));
+          }
+        }
+      }
+      pend_n = 0;
+    }
+  }
+  if (pend_n) {                                    // the last tile's survivors
+    if (tid == 0) {
+      s_base[par ^ 1] = pend_base;
+      seg[(uint64_t)pend_row * n_tiles + pend_t] = make_uint2(pend_base, pend_n);
+    }
+    __syncthreads();
+    const uint32_t base = s_base[par ^ 1];
+    uint2* out = cand + (uint64_t)pend_row * cap;
+    for (uint32_t i = tid; i < pend_n; i += kTileThreads)
+      if (base + i < cap) out[base + i] = s_stage[par ^ 1][i];
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
@@ -306,7 +406,10 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   count_launch(2);
   uint64_t n_work = (uint64_t)L.M * L.n_tiles;
   uint64_t blocks = n_work < (uint64_t)kSMs * 8 ? n_work : (uint64_t)kSMs * 8;
-  filter_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
+  if ((uint64_t)L.typical_cand * 250u > L.d)
+    filter_scan_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
+  else
+    filter_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
   return cudaGetLastError();
 }
 
