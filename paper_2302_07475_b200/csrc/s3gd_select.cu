@@ -128,18 +128,25 @@ __global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* 
   const uint32_t mask = (uint32_t)(nbins - 1);
   uint32_t* g_hist = hist + (uint64_t)row * kHistBins;
   bool worked = false;
-  if (is_c && use_c && (uint64_t)blockIdx.x * kSelThreads < rs.n_cand) {
+  if (is_c && use_c && (uint64_t)blockIdx.x * kSelThreads * 4 < rs.n_cand) {
     worked = true;
     for (int b = threadIdx.x; b < nbins; b += kSelThreads) s_hist[b] = 0u;
     __syncthreads();
     const uint2* c = cand + (uint64_t)row * cap;
-    const uint32_t n = rs.n_cand, step = gx_c * kSelThreads;
-    const uint32_t n_round = (n + 31u) & ~31u;        // whole warps stay in the loop together
-    for (uint32_t i = blockIdx.x * kSelThreads + threadIdx.x; i < n_round; i += step) {
-      bool on = i < n;
-      const uint32_t key = on ? (c[i].x & kAbsMask) : 0u;
-      on = on && in_prefix(key, rs.prefix, pass);
-      hist_add(s_hist, on, (key >> pass_shift(pass)) & mask);
+    // four entries per thread and round, all four loads issued before the first is used
+    const uint32_t n = rs.n_cand, step = gx_c * kSelThreads * 4;
+    for (uint32_t base = blockIdx.x * kSelThreads * 4; base < n; base += step) {
+      uint32_t key[4];
+      bool on[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t i = base + u * kSelThreads + threadIdx.x;
+        on[u] = i < n;
+        key[u] = on[u] ? (c[i].x & kAbsMask) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        hist_add(s_hist, on[u] && in_prefix(key[u], rs.prefix, pass), (key[u] >> pass_shift(pass)) & mask);
     }
   } else if (!is_c && !use_c) {
     worked = true;

@@ -12,14 +12,26 @@ __device__ __forceinline__ void count_cand(const uint2* __restrict__ cand, uint3
   const uint32_t lane = threadIdx.x & 31;
   const uint32_t warps = gx * (kSelThreads >> 5);
   const uint2* c = cand + (uint64_t)row * cap;
-  for (uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
-    const uint2 sg = seg[(uint64_t)row * n_tiles + t];
+  const uint2* sgp = seg + (uint64_t)row * n_tiles;
+  uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5);
+  uint2 sg_next = t < n_tiles ? sgp[t] : make_uint2(0u, 0u);
+  for (; t < n_tiles; t += warps) {
+    const uint2 sg = sg_next;
+    if (t + warps < n_tiles) sg_next = sgp[t + warps];        // next tile's segment is on its way meanwhile
     uint32_t gt = 0, eq = 0;
-    for (uint32_t i0 = 0; i0 < sg.y; i0 += 32) {
-      const uint32_t i = i0 + lane;
-      const uint32_t key = (i < sg.y) ? (c[sg.x + i].x & kAbsMask) : 0u;
-      gt += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key > rs.tau));
-      eq += __popc(__ballot_sync(0xFFFFFFFFu, i < sg.y && key == rs.tau));
+    for (uint32_t i0 = 0; i0 < sg.y; i0 += 128) {             // four 32-entry loads in flight
+      uint32_t key[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t i = i0 + u * 32 + lane;
+        key[u] = i < sg.y ? (c[sg.x + i].x & kAbsMask) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool in = i0 + u * 32 + lane < sg.y;
+        gt += __popc(__ballot_sync(0xFFFFFFFFu, in && key[u] > rs.tau));
+        eq += __popc(__ballot_sync(0xFFFFFFFFu, in && key[u] == rs.tau));
+      }
     }
     if (lane == 0) cnt[(uint64_t)row * n_tiles + t] = make_uint2(gt, eq);
   }
@@ -96,21 +108,37 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* s
 __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles, RowState* __restrict__ rows,
                                          uint32_t row, uint32_t K, uint32_t cap, uint32_t* __restrict__ hdr,
                                          uint32_t* s_warp) {
+  constexpr int kPer = 8;                            // consecutive tiles per thread and round
   const uint32_t tid = threadIdx.x;
   const uint32_t take = rows[row].take_ties;
   uint32_t carry_eq = 0, carry_out = 0;
-  uint2 next = tid < n_tiles ? __ldcg(&c[tid]) : make_uint2(0u, 0u);
-  for (uint32_t base = 0; base < n_tiles; base += kSelThreads) {     // kSelThreads tiles per round, next round in flight
-    const uint32_t t = base + tid;
-    const uint2 v = next;
-    const uint32_t tn = t + kSelThreads;
-    next = tn < n_tiles ? __ldcg(&c[tn]) : make_uint2(0u, 0u);
+  for (uint32_t base = 0; base < n_tiles; base += kSelThreads * kPer) {
+    const uint32_t t0 = base + tid * kPer;
+    uint2 v[kPer];
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) v[q] = t0 + q < n_tiles ? __ldcg(&c[t0 + q]) : make_uint2(0u, 0u);
+    uint32_t eq_sum = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) eq_sum += v[q].y;
     uint32_t tot_eq, tot_sel;
-    const uint32_t run_eq = carry_eq + block_exclusive_scan(v.y, s_warp, &tot_eq);
-    const uint32_t room = run_eq < take ? take - run_eq : 0u;
-    const uint32_t sel = v.x + (v.y < room ? v.y : room);
-    const uint32_t out = carry_out + block_exclusive_scan(sel, s_warp, &tot_sel);
-    if (t < n_tiles) c[t] = make_uint2(out, run_eq);
+    uint32_t run_eq = carry_eq + block_exclusive_scan(eq_sum, s_warp, &tot_eq);
+    const uint32_t eq0 = run_eq;
+    uint32_t sel_sum = 0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const uint32_t room = run_eq < take ? take - run_eq : 0u;
+      sel_sum += v[q].x + (v[q].y < room ? v[q].y : room);
+      run_eq += v[q].y;
+    }
+    uint32_t out = carry_out + block_exclusive_scan(sel_sum, s_warp, &tot_sel);
+    run_eq = eq0;
+#pragma unroll
+    for (int q = 0; q < kPer; ++q) {
+      const uint32_t room = run_eq < take ? take - run_eq : 0u;
+      if (t0 + q < n_tiles) c[t0 + q] = make_uint2(out, run_eq);
+      out += v[q].x + (v[q].y < room ? v[q].y : room);
+      run_eq += v[q].y;
+    }
     carry_eq += tot_eq;
     carry_out += tot_sel;
   }
@@ -157,38 +185,51 @@ __device__ __forceinline__ void emit_cand(const uint2* __restrict__ cand, uint32
   const uint32_t lane = threadIdx.x & 31, lt = lanemask_lt();
   const uint32_t warps = gx * (kSelThreads >> 5);
   const uint2* c = cand + (uint64_t)row * cap;
-  for (uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5); t < n_tiles; t += warps) {
-    const uint2 sg = seg[(uint64_t)row * n_tiles + t];
-    if (sg.y == 0) continue;
-    const uint2 sc = scan[(uint64_t)row * n_tiles + t];
+  const uint2* sgp = seg + (uint64_t)row * n_tiles;
+  const uint2* scp = scan + (uint64_t)row * n_tiles;
+  uint32_t t = bx * (kSelThreads >> 5) + (threadIdx.x >> 5);
+  uint2 sg_next = make_uint2(0u, 0u), sc_next = make_uint2(0u, 0u);
+  if (t < n_tiles) { sg_next = sgp[t]; sc_next = scp[t]; }
+  for (; t < n_tiles; t += warps) {
+    const uint2 sg = sg_next, sc = sc_next;
+    if (t + warps < n_tiles) { sg_next = sgp[t + warps]; sc_next = scp[t + warps]; }   // in flight meanwhile
     uint32_t run_out = sc.x, run_eq = sc.y;
-    for (uint32_t i0 = 0; i0 < sg.y; i0 += 32) {
-      const uint32_t i = i0 + lane;
-      const bool in = i < sg.y;
-      uint2 e = in ? c[sg.x + i] : make_uint2(0u, 0u);
-      const uint32_t key = e.x & kAbsMask;
-      const bool eq = in && key == rs.tau;
-      const uint32_t eqb = __ballot_sync(0xFFFFFFFFu, eq);
-      const bool sel = in && (key > rs.tau || (eq && run_eq + __popc(eqb & lt) < rs.take_ties));
-      const uint32_t selb = __ballot_sync(0xFFFFFFFFu, sel);
-      const uint32_t pos = run_out + __popc(selb & lt);
-      const uint32_t neg = e.x >> 31;
-      if (sel && pos < o.K) {
-        if (o.idx) o.idx[(uint64_t)row * o.K + pos] = e.y;
-        if (o.counter) atomicAdd(o.counter + e.y, neg ? -1 : 1);
+    for (uint32_t i0 = 0; i0 < sg.y; i0 += 128) {             // four 32-entry loads in flight
+      uint2 ent[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t i = i0 + u * 32 + lane;
+        ent[u] = i < sg.y ? c[sg.x + i] : make_uint2(0u, 0u);
       }
-      if (o.signbits && selb) {
-        const uint32_t w0 = run_out >> 5;
-        const uint32_t bit = (sel && pos < o.K) ? (neg << (pos & 31)) : 0u;
-        const uint32_t v0 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 ? bit : 0u);
-        const uint32_t v1 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 + 1 ? bit : 0u);
-        if (lane == 0) {
-          if (v0) atomicOr(o.signbits + (uint64_t)row * o.words + w0, v0);
-          if (v1) atomicOr(o.signbits + (uint64_t)row * o.words + w0 + 1, v1);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (i0 + u * 32 >= sg.y) break;                        // warp-uniform
+        const bool in = i0 + u * 32 + lane < sg.y;
+        const uint2 e = ent[u];
+        const uint32_t key = e.x & kAbsMask;
+        const bool eq = in && key == rs.tau;
+        const uint32_t eqb = __ballot_sync(0xFFFFFFFFu, eq);
+        const bool sel = in && (key > rs.tau || (eq && run_eq + __popc(eqb & lt) < rs.take_ties));
+        const uint32_t selb = __ballot_sync(0xFFFFFFFFu, sel);
+        const uint32_t pos = run_out + __popc(selb & lt);
+        const uint32_t neg = e.x >> 31;
+        if (sel && pos < o.K) {
+          if (o.idx) o.idx[(uint64_t)row * o.K + pos] = e.y;
+          if (o.counter) atomicAdd(o.counter + e.y, neg ? -1 : 1);
         }
+        if (o.signbits && selb) {
+          const uint32_t w0 = run_out >> 5;
+          const uint32_t bit = (sel && pos < o.K) ? (neg << (pos & 31)) : 0u;
+          const uint32_t v0 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 ? bit : 0u);
+          const uint32_t v1 = __reduce_or_sync(0xFFFFFFFFu, (pos >> 5) == w0 + 1 ? bit : 0u);
+          if (lane == 0) {
+            if (v0) atomicOr(o.signbits + (uint64_t)row * o.words + w0, v0);
+            if (v1) atomicOr(o.signbits + (uint64_t)row * o.words + w0 + 1, v1);
+          }
+        }
+        run_out += __popc(selb);
+        run_eq += __popc(eqb);
       }
-      run_out += __popc(selb);
-      run_eq += __popc(eqb);
     }
   }
 }
