@@ -110,7 +110,7 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
 }
 
 // grid (gx_c + gx_r, M): the first gx_c blocks of a row walk its candidates, the others its tiles.
-__global__ void __launch_bounds__(kSelThreads) hist_pick_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+__global__ void __launch_bounds__(kSelThreads, 6) hist_pick_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 uint32_t n_tiles, const uint2* __restrict__ cand,
                                                                 uint32_t cap, RowState* __restrict__ rows, uint32_t K,
                                                                 uint32_t* __restrict__ hist,

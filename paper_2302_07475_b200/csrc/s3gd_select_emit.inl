@@ -155,7 +155,7 @@ __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles
 }
 
 // grid (gx_c + gx_r, M)
-__global__ void __launch_bounds__(kSelThreads) count_scan_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+__global__ void __launch_bounds__(kSelThreads, 6) count_scan_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                  uint32_t n_tiles, const uint2* __restrict__ cand,
                                                                  uint32_t cap, const uint2* __restrict__ seg,
                                                                  RowState* __restrict__ rows, uint32_t K,
@@ -322,7 +322,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
 }
 
 // grid (gx_c + gx_r, M)
-__global__ void __launch_bounds__(kSelThreads) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+__global__ void __launch_bounds__(kSelThreads, 6) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                            uint32_t n_tiles, const uint2* __restrict__ cand,
                                                            uint32_t cap, const uint2* __restrict__ seg,
                                                            const uint2* __restrict__ scan,
