@@ -124,6 +124,33 @@ S3GD_API s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, 
                       void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The step with the two optional parts of Algorithm 1 around it:
+ *
+ *  - error compensation (Section 2.2, Eq. (5)-(6)), if opt_err != NULL: the selection works on
+ *    g = grads + eta * err (fp32: the product rounded, then the sum rounded); afterwards err
+ *    holds g with its K kept entries per worker set to +0, i.e. g - TopK(g);
+ *  - momentum (Section 4.7), if opt_v != NULL: v <- mu * v + vote, x <- x - lr * v (every
+ *    operation rounded once) instead of x <- x - lr * vote.  v and x change at every coordinate.
+ *
+ *  grads    dev, const [M x d]  this iteration's stochastic gradients (g~)
+ *  opt_err  dev or NULL [M x d]  error memory e, updated in place (all zero before the first step)
+ *  opt_v    dev or NULL [d]      momentum v, updated in place
+ *  everything else as for s3gd_step.  With both NULL the call is s3gd_step.
+ *  K == d with error memory leaves err all zero (everything is kept); K == 0 leaves err = g.
+ */
+S3GD_API s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta, float* opt_v, float mu,
+                                  int M, uint64_t d, uint64_t K, float lr,
+                                  uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Momentum form of the update for the unfused route (Section 4.7): v[n] <- fl(fl(mu * v[n]) + sgn(vote[n])),
+ * x[n] <- fl(x[n] - fl(lr * v[n])).  x, v dev [d] fp32 in place; vote dev, const [d] int8.
+ */
+S3GD_API s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
+                                         void* stream);
+
+/*
  * Waits for `stream`, then reports what the kernels of earlier calls on this
  * workspace recorded: S3GD_OK, S3GD_ERR_INDEX_RANGE or S3GD_ERR_INTERNAL.
  * The record is cleared by the next s3gd_topk_sign / s3gd_majority_vote / s3gd_step.

@@ -26,6 +26,8 @@ Readings where the paper is silent (all listed in the design notes):
 * the update is one fp32 round-to-nearest operation: x - lr or x + lr.
 
 All integer results are exact, so GPU output must equal them bit for bit.
+Also here: error compensation (Eq. (5)-(6)) and the momentum update (Section 4.7).
+
 Parity status: every function below is pinned by tests that do not call it to
 build their expectation (brute-force rank counting, the printed worked
 example, the K = N and M = 1 special cases of Section 3.3, invariants).
@@ -134,6 +136,49 @@ def step(x: np.ndarray, grads: np.ndarray, K: int, lr):
     idx, sgn = topk_sign(grads, K)
     vote, _ = majority_vote(idx, sgn, M, K, d)
     return apply_vote(x, vote, lr), idx, sgn, vote
+
+
+# --------------------------------------------------------------------------
+# The lines of Algorithm 1 around the step: error compensation before it
+# (Section 2.2, Eq. (5)-(6)) and the momentum form of the update after it
+# (Section 4.7, the two displays that replace Eq. (7)).
+# --------------------------------------------------------------------------
+
+def error_feedback_step(x, grads_tilde, err, eta, K: int, lr, topk=None):
+    """Algorithm 1 with error memory, one iteration for all workers.
+
+    g_m = g~_m + eta * e_m            (Eq. (5); fp32: one rounding for the product, one for the sum)
+    e_m <- g_m - TopK(g_m)            (Eq. (6): g_m with its K kept entries set to zero)
+    x   <- x - lr * sgn(sum_m TopKSign(g_m))
+
+    Returns (x_new, err_new, idx, signbits, vote).  TopK(g) keeps the values of the K
+    selected entries, so err_new equals g off the support and is exactly +0 on it.
+    """
+    gt = np.asarray(grads_tilde, dtype=np.float32)
+    e = np.asarray(err, dtype=np.float32)
+    M, d = gt.shape
+    eta32 = np.float32(eta)
+    g = (gt + (eta32 * e).astype(np.float32)).astype(np.float32)
+    idx, sgn = (topk or topk_sign)(g, K)
+    vote, _ = majority_vote(idx, sgn, M, K, d)
+    err_new = g.copy()
+    for m in range(M):
+        err_new[m][idx[m].astype(np.int64)] = np.float32(0.0)
+    return apply_vote(x, vote, lr), err_new, idx, sgn, vote
+
+
+def apply_vote_momentum(x, v, vote, mu, lr):
+    """Momentum form of the update (Section 4.7): v <- mu * v + vote ; x <- x - lr * v.
+
+    fp32 with one rounding per operation: fl(mu*v), fl(. + vote), fl(lr*v), fl(x - .).
+    Returns (x_new, v_new).
+    """
+    x = np.asarray(x, dtype=np.float32)
+    v = np.asarray(v, dtype=np.float32)
+    mu32, lr32 = np.float32(mu), np.float32(lr)
+    v_new = ((mu32 * v).astype(np.float32) + np.asarray(vote).astype(np.float32)).astype(np.float32)
+    x_new = (x - (lr32 * v_new).astype(np.float32)).astype(np.float32)
+    return x_new, v_new
 
 
 # --------------------------------------------------------------------------

@@ -24,7 +24,7 @@ STATUS_NAMES = {
 
 EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
            "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
-           "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc")
+           "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum")
 
 
 class S3gdError(RuntimeError):
@@ -70,6 +70,11 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_noalloc_max_d.argtypes = []
     lib.s3gd_majority_vote_noalloc.restype = ctypes.c_int
     lib.s3gd_majority_vote_noalloc.argtypes = [u32p, u32p, ctypes.c_int, u64, u64, vp, vp, vp]
+    lib.s3gd_step_ex.restype = ctypes.c_int
+    lib.s3gd_step_ex.argtypes = [vp, vp, vp, ctypes.c_float, vp, ctypes.c_float, ctypes.c_int, u64, u64, ctypes.c_float,
+                                 u32p, u32p, vp, vp, sz, vp]
+    lib.s3gd_apply_momentum.restype = ctypes.c_int
+    lib.s3gd_apply_momentum.argtypes = [vp, vp, vp, u64, ctypes.c_float, ctypes.c_float, vp]
     if path is None:
         _lib = lib
     return lib
@@ -204,3 +209,30 @@ def s3gd_majority_vote_noalloc(idx: torch.Tensor, signbits: torch.Tensor, M: int
     with torch.cuda.device(out_vote.device):
         code = load().s3gd_majority_vote_noalloc(*args, _stream(out_vote))
     _check("s3gd_majority_vote_noalloc", code)
+
+
+def s3gd_step_ex(x: torch.Tensor, grads: torch.Tensor, K: int, lr: float, ws: torch.Tensor,
+                 err: Optional[torch.Tensor] = None, eta: float = 1.0,
+                 v: Optional[torch.Tensor] = None, mu: float = 0.0,
+                 opt_idx: Optional[torch.Tensor] = None, opt_signbits: Optional[torch.Tensor] = None,
+                 opt_vote: Optional[torch.Tensor] = None) -> None:
+    """The fused step with optional error memory err [M, d] (updated in place) and momentum v [d]."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (_ptr(x, torch.float32, d, "x"), g, _ptr(err, torch.float32, M * d, "err"), ctypes.c_float(eta),
+            _ptr(v, torch.float32, d, "v"), ctypes.c_float(mu), M, d, K, ctypes.c_float(lr),
+            _ptr(opt_idx, torch.int32, M * K, "opt_idx"), _ptr(opt_signbits, torch.int32, M * words(K), "opt_signbits"),
+            _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(x.device):
+        code = load().s3gd_step_ex(*args, _stream(x))
+    _check("s3gd_step_ex", code)
+
+
+def s3gd_apply_momentum(x: torch.Tensor, v: torch.Tensor, vote: torch.Tensor, mu: float, lr: float) -> None:
+    """v <- mu * v + vote; x <- x - lr * v, in place."""
+    d = x.numel()
+    args = (_ptr(x, torch.float32, name="x"), _ptr(v, torch.float32, d, "v"), _ptr(vote, torch.int8, d, "vote"), d,
+            ctypes.c_float(mu), ctypes.c_float(lr))
+    with torch.cuda.device(x.device):
+        code = load().s3gd_apply_momentum(*args, _stream(x))
+    _check("s3gd_apply_momentum", code)

@@ -138,7 +138,7 @@ s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, ui
     return S3GD_OK;
   }
   S3GD_TRY(cudaMemsetAsync(out_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, st));
+  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, nullptr, st));
 }
 
 s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
@@ -165,37 +165,93 @@ s3gd_status s3gd_apply(float* x, const int8_t* vote, uint64_t d, float lr, void*
   return from_cuda(launch_apply(x, vote, d, lr, static_cast<cudaStream_t>(stream)));
 }
 
-s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
-                      uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
-  Layout L;
-  if (!make_layout(M, d, K, &L) || x == nullptr || grads == nullptr || !aligned(x, 4) || !aligned(grads, 4))
-    return S3GD_ERR_INVALID_ARG;
-  if ((opt_idx == nullptr) != (opt_signbits == nullptr)) return S3GD_ERR_INVALID_ARG;
-  if (opt_idx != nullptr && (!aligned(opt_idx, 4) || !aligned(opt_signbits, 4))) return S3GD_ERR_INVALID_ARG;
-  s3gd_status s = check_ws(L, ws, ws_bytes);
-  if (s != S3GD_OK) return s;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+namespace {
+
+// The step on `sel` (the gradients the selection looks at).  err_to_clear: error memory whose kept
+// entries are zeroed (it is `sel` itself when error compensation is on).  v: momentum buffer or NULL.
+s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v, float mu, int M, uint64_t d,
+                      uint64_t K, float lr, uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
+                      const Layout& L, void* ws, cudaStream_t st) {
   char* base = static_cast<char*>(ws);
+  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
   if (K == 0 || K == d) {
     S3GD_TRY(cudaMemsetAsync(base + L.off_hdr, 0, kHdrWords * sizeof(uint32_t), st));
+    for (int ph = kPhaseStart; ph < kPhaseApplied; ++ph) prof_mark(ph, st);
     if (K == 0) {
       if (opt_vote) S3GD_TRY(cudaMemsetAsync(opt_vote, 0, (size_t)d, st));
+      if (v) {                                 // no votes, but the momentum still decays and moves x
+        S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+        S3GD_TRY(launch_counter_apply_momentum(counter, x, v, d, mu, lr, nullptr, st));
+      }
+      prof_mark(kPhaseApplied, st);
       return S3GD_OK;
     }
-    if (opt_idx) S3GD_TRY(launch_signplane_message(grads, M, d, opt_idx, opt_signbits, st));
-    for (int ph = kPhaseStart; ph < kPhaseApplied; ++ph) prof_mark(ph, st);
-    cudaError_t e = launch_signplane_step(x, grads, M, d, lr, opt_vote, st);
+    if (opt_idx) S3GD_TRY(launch_signplane_message(sel, M, d, opt_idx, opt_signbits, st));
+    if (v) {
+      S3GD_TRY(launch_signplane_counts(sel, M, d, counter, st));
+      S3GD_TRY(launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st));
+    } else {
+      S3GD_TRY(launch_signplane_step(x, sel, M, d, lr, opt_vote, st));
+    }
+    if (err_to_clear) S3GD_TRY(cudaMemsetAsync(err_to_clear, 0, (size_t)M * d * sizeof(float), st));   // everything was kept
     prof_mark(kPhaseApplied, st);
-    return from_cuda(e);
+    return S3GD_OK;
   }
-  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
   prof_mark(kPhaseStart, st);
   S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  S3GD_TRY(launch_select(grads, L, ws, opt_idx, opt_signbits, counter, st));
-  cudaError_t e = launch_counter_apply(counter, x, d, lr, opt_vote, st);
+  S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, st));
+  cudaError_t e = v ? launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st)
+                    : launch_counter_apply(counter, x, d, lr, opt_vote, st);
   prof_mark(kPhaseApplied, st);
   return from_cuda(e);
+}
+
+s3gd_status check_step_args(const float* x, const float* grads, uint32_t* opt_idx, uint32_t* opt_signbits) {
+  if (x == nullptr || grads == nullptr || !aligned(x, 4) || !aligned(grads, 4)) return S3GD_ERR_INVALID_ARG;
+  if ((opt_idx == nullptr) != (opt_signbits == nullptr)) return S3GD_ERR_INVALID_ARG;
+  if (opt_idx != nullptr && (!aligned(opt_idx, 4) || !aligned(opt_signbits, 4))) return S3GD_ERR_INVALID_ARG;
+  return S3GD_OK;
+}
+
+}  // namespace
+
+s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
+                      uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L)) return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_step_args(x, grads, opt_idx, opt_signbits);
+  if (s != S3GD_OK) return s;
+  s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  return step_impl(x, grads, nullptr, nullptr, 0.f, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws,
+                   static_cast<cudaStream_t>(stream));
+}
+
+s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta, float* opt_v, float mu, int M,
+                         uint64_t d, uint64_t K, float lr, uint32_t* opt_idx, uint32_t* opt_signbits,
+                         int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L)) return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_step_args(x, grads, opt_idx, opt_signbits);
+  if (s != S3GD_OK) return s;
+  if ((opt_err != nullptr && !aligned(opt_err, 4)) || (opt_v != nullptr && !aligned(opt_v, 4))) return S3GD_ERR_INVALID_ARG;
+  s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float* sel = grads;
+  if (opt_err != nullptr) {                    // g = g~ + eta * e, kept in the error memory
+    S3GD_TRY(launch_ef_accumulate(opt_err, grads, eta, (uint64_t)M * d, st));
+    sel = opt_err;
+  }
+  return step_impl(x, sel, opt_err, opt_v, mu, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws, st);
+}
+
+s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
+                                void* stream) {
+  if (x == nullptr || v == nullptr || vote == nullptr || d == 0 || d >= (1ull << 32) || !aligned(x, 4) || !aligned(v, 4))
+    return S3GD_ERR_INVALID_ARG;
+  return from_cuda(launch_apply_momentum(x, v, vote, d, mu, lr, static_cast<cudaStream_t>(stream)));
 }
 
 s3gd_status s3gd_profile_begin(int max_steps) {

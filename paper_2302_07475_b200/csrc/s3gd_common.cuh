@@ -136,6 +136,8 @@ struct EmitOut {
   uint32_t* idx;        // [M x K] or NULL
   uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
   int32_t* counter;     // [d] or NULL
+  float* err;           // [M x d] or NULL: error memory whose kept entries are set to zero (Eq. (6))
+  uint64_t d;
   uint32_t K, words;
 };
 cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* cand, const uint2* seg, uint32_t* hdr,
@@ -143,6 +145,15 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, cudaStream_t st);
+                          int32_t* counter, float* err_to_clear, cudaStream_t st);
+// err <- grads + eta * err, element-wise over n entries (Eq. (5))
+cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint64_t n, cudaStream_t st);
+// v <- mu * v + sgn(counter); x <- x - lr * v (momentum form of the update)
+cudaError_t launch_counter_apply_momentum(const int32_t* counter, float* x, float* v, uint64_t d, float mu, float lr,
+                                          int8_t* opt_vote, cudaStream_t st);
+cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
+                                  cudaStream_t st);
+// counter[n] <- sum over workers of (+1 | -1) by sign bit (K = d, when the sign counts are needed as such)
+cudaError_t launch_signplane_counts(const float* grads, int M, uint64_t d, int32_t* counter, cudaStream_t st);
 
 }  // namespace s3gd

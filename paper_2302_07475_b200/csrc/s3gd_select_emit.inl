@@ -216,6 +216,7 @@ __device__ __forceinline__ void emit_cand(const uint2* __restrict__ cand, uint32
         if (sel && pos < o.K) {
           if (o.idx) o.idx[(uint64_t)row * o.K + pos] = e.y;
           if (o.counter) atomicAdd(o.counter + e.y, neg ? -1 : 1);
+          if (o.err) o.err[(uint64_t)row * o.d + e.y] = 0.f;
         }
         if (o.signbits && selb) {
           const uint32_t w0 = run_out >> 5;
@@ -282,6 +283,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
       if (pos < o.K) {
         if (o.idx) o.idx[(uint64_t)row * o.K + pos] = lane;
         if (o.counter) atomicAdd(o.counter + lane, neg ? -1 : 1);
+        if (o.err) o.err[(uint64_t)row * o.d + lane] = 0.f;
         if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
       }
     }
@@ -300,6 +302,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
             const uint32_t neg = T.bits[it][q] >> 31;
             if (o.idx) o.idx[(uint64_t)row * o.K + pos] = n;
             if (o.counter) atomicAdd(o.counter + n, neg ? -1 : 1);
+            if (o.err) o.err[(uint64_t)row * o.d + n] = 0.f;
             const uint32_t rel = (pos >> 5) - (p0 >> 5);      // 0..4: at most 128 entries per warp-iteration
 #pragma unroll
             for (int w = 0; w < 5; ++w)
@@ -322,7 +325,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
 }
 
 // grid (gx_c + gx_r, M)
-__global__ void __launch_bounds__(kSelThreads, 6) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+__global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                            uint32_t n_tiles, const uint2* __restrict__ cand,
                                                            uint32_t cap, const uint2* __restrict__ seg,
                                                            const uint2* __restrict__ scan,
@@ -343,7 +346,7 @@ inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)
 }  // namespace
 
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, cudaStream_t st) {
+                          int32_t* counter, float* err_to_clear, cudaStream_t st) {
   char* base = static_cast<char*>(ws);
   uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
   RowState* rows = reinterpret_cast<RowState*>(base + L.off_rows);
@@ -373,6 +376,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   prof_mark(kPhaseFiltered, st);
   EmitOut o;
   o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
+  o.err = err_to_clear; o.d = L.d;
   o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
   if (use_filter) {                                  // rows whose candidates fit one SM are finished here
     cudaError_t e = launch_select_small(L, rows, cand, seg, hdr, o, st);

@@ -201,7 +201,9 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     for (uint32_t i = tid; i < n; i += kSmallThreads) {
       const uint32_t bits = s_bits[i], key = bits & kAbsMask;
       if (key > tau || (key == tau && !rank_ties)) {
-        atomicAdd(o.counter + s_idx[i], (bits >> 31) ? -1 : 1);
+        const uint32_t idx = s_idx[i];
+        atomicAdd(o.counter + idx, (bits >> 31) ? -1 : 1);
+        if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
       } else if (key == tau) {
         const uint32_t slot = atomicAdd(&s_sel[0], 1u);
         s_tie_idx[slot] = s_idx[i];
@@ -216,7 +218,10 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
         const uint32_t mine = s_tie_idx[tid];
         uint32_t before = 0;
         for (uint32_t j = 0; j < e; ++j) before += (uint32_t)(s_tie_idx[j] < mine);
-        if (before < take) atomicAdd(o.counter + mine, s_tie_neg[tid] ? -1 : 1);
+        if (before < take) {
+          atomicAdd(o.counter + mine, s_tie_neg[tid] ? -1 : 1);
+          if (o.err) o.err[(uint64_t)row * o.d + mine] = 0.f;
+        }
       }
       if (e != n_equal) n_kept = 0xFFFFFFFFu;                    // cannot happen
     }
@@ -270,6 +275,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
           const uint32_t neg = bits[q] >> 31;
           if (o.idx) o.idx[(uint64_t)row * o.K + pos] = idx;
           if (o.counter) atomicAdd(o.counter + idx, neg ? -1 : 1);
+          if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
           // sign bits only when the message is asked for: one atomic per negative entry
           if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
         }

@@ -87,6 +87,17 @@ __global__ void __launch_bounds__(256) signplane_message_kernel(const float* __r
   }
 }
 
+// Sign counts only: counter[n] = sum over workers of (+1 | -1).
+__global__ void __launch_bounds__(256) signplane_counts_kernel(const float* __restrict__ grads, int M, uint64_t d,
+                                                               int32_t* __restrict__ counter) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+    int negs = 0;
+    for (int m = 0; m < M; ++m) negs += (int)(ld_stream_u32(grads + (uint64_t)m * d + n) >> 31);
+    counter[n] = M - 2 * negs;
+  }
+}
+
 inline unsigned blocks_for(uint64_t threads) {
   uint64_t b = (threads + 255) / 256;
   uint64_t cap = (uint64_t)kSMs * 8;
@@ -116,6 +127,12 @@ cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint
                                      uint32_t* out_signbits, cudaStream_t st) {
   uint64_t warps = (uint64_t)M * ((d + 31) / 32);
   signplane_message_kernel<<<blocks_for(warps * 32), 256, 0, st>>>(grads, M, d, out_idx, out_signbits);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_signplane_counts(const float* grads, int M, uint64_t d, int32_t* counter, cudaStream_t st) {
+  signplane_counts_kernel<<<blocks_for(d), 256, 0, st>>>(grads, M, d, counter);
   count_launch();
   return cudaGetLastError();
 }

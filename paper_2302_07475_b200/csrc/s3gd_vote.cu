@@ -118,6 +118,61 @@ __global__ void __launch_bounds__(256) counter_apply_kernel(const int32_t* __res
   }
 }
 
+// err <- grads + eta * err: one rounding for the product, one for the sum (Eq. (5))
+__global__ void __launch_bounds__(256) ef_accumulate_kernel(float* __restrict__ err, const float* __restrict__ grads,
+                                                            float eta, uint64_t n) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    err[i] = __fadd_rn(grads[i], __fmul_rn(eta, err[i]));
+}
+
+__global__ void __launch_bounds__(256) ef_accumulate_kernel_v4(float4* __restrict__ err, const float4* __restrict__ grads,
+                                                               float eta, uint64_t n4) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const float4 g = grads[i];
+    float4 e = err[i];
+    e.x = __fadd_rn(g.x, __fmul_rn(eta, e.x));
+    e.y = __fadd_rn(g.y, __fmul_rn(eta, e.y));
+    e.z = __fadd_rn(g.z, __fmul_rn(eta, e.z));
+    e.w = __fadd_rn(g.w, __fmul_rn(eta, e.w));
+    err[i] = e;
+  }
+}
+
+// Momentum form of the update: v <- mu * v + s ; x <- x - lr * v, every operation rounded once.
+__device__ __forceinline__ void momentum_update(float& x, float& v, int s, float mu, float lr) {
+  v = __fadd_rn(__fmul_rn(mu, v), (float)((s > 0) - (s < 0)));
+  x = __fsub_rn(x, __fmul_rn(lr, v));
+}
+
+__global__ void __launch_bounds__(256) counter_apply_momentum_kernel(const int32_t* __restrict__ counter,
+                                                                     float* __restrict__ x, float* __restrict__ v,
+                                                                     uint64_t d, float mu, float lr,
+                                                                     int8_t* __restrict__ opt_vote) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+    const int c = counter[n];
+    if (opt_vote) opt_vote[n] = (int8_t)((c > 0) - (c < 0));
+    float xv = x[n], vv = v[n];
+    momentum_update(xv, vv, c, mu, lr);
+    x[n] = xv;
+    v[n] = vv;
+  }
+}
+
+__global__ void __launch_bounds__(256) apply_momentum_kernel(float* __restrict__ x, float* __restrict__ v,
+                                                             const int8_t* __restrict__ vote, uint64_t d, float mu,
+                                                             float lr) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
+    float xv = x[n], vv = v[n];
+    momentum_update(xv, vv, vote[n], mu, lr);
+    x[n] = xv;
+    v[n] = vv;
+  }
+}
+
 inline unsigned grid_for(uint64_t items, int per_block, int max_blocks) {
   uint64_t b = (items + per_block - 1) / per_block;
   if (b < 1) b = 1;
@@ -169,6 +224,37 @@ cudaError_t launch_counter_apply(const int32_t* counter, float* x, uint64_t d, f
     counter_apply_kernel<false><<<grid_for(d, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
     count_launch();
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint64_t n, cudaStream_t st) {
+  if (aligned(err, 16) && aligned(grads, 16) && n >= 4) {
+    const uint64_t n4 = n / 4;
+    ef_accumulate_kernel_v4<<<grid_for(n4, 256, kSMs * 16), 256, 0, st>>>(reinterpret_cast<float4*>(err),
+                                                                         reinterpret_cast<const float4*>(grads), eta, n4);
+    count_launch();
+    if (n4 * 4 < n) {
+      ef_accumulate_kernel<<<1, 256, 0, st>>>(err + n4 * 4, grads + n4 * 4, eta, n - n4 * 4);
+      count_launch();
+    }
+  } else {
+    ef_accumulate_kernel<<<grid_for(n, 256, kSMs * 16), 256, 0, st>>>(err, grads, eta, n);
+    count_launch();
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_counter_apply_momentum(const int32_t* counter, float* x, float* v, uint64_t d, float mu, float lr,
+                                          int8_t* opt_vote, cudaStream_t st) {
+  counter_apply_momentum_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
+                                  cudaStream_t st) {
+  apply_momentum_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(x, v, vote, d, mu, lr);
+  count_launch();
   return cudaGetLastError();
 }
 

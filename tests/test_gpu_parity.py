@@ -277,6 +277,70 @@ def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
     assert info[1] == 0                      # no row fell back to the whole-row route
 
 
+# ------------------------------------------- error compensation and momentum (s3gd_step_ex)
+@pytest.mark.parametrize("K,eta,mu", [(300, 1.0, None), (300, 0.5, 0.9), (75_002, 1.0, None), (300_007, 1.0, 0.5),
+                                      (0, 1.0, 0.5), (3_000, 0.0, None)])
+def test_error_memory_and_momentum_over_steps(K, eta, mu):
+    """Four consecutive steps with carried state: x, the error memory e and the momentum v must
+    equal the oracle's bit for bit after every step, as must the message and the vote."""
+    s = W.spec("small_cnn", d=300_007, M=6)
+    d, M = s.d, s.M
+    x = W.make_x(s, DEV)
+    err = torch.zeros((M, d), device=DEV)
+    v = torch.zeros(d, device=DEV) if mu is not None else None
+    x_o, e_o = x.cpu().numpy(), np.zeros((M, d), np.float32)
+    v_o = np.zeros(d, np.float32)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    idx = torch.empty((M, max(K, 1)), dtype=torch.int32, device=DEV)[:, :K].contiguous()
+    sgn = torch.empty((M, max(S.binding.words(K), 1)), dtype=torch.int32, device=DEV)[:, :S.binding.words(K)].contiguous()
+    vote = torch.empty(d, dtype=torch.int8, device=DEV)
+    for step in range(4):
+        g = W.make_grads(s, DEV, step=step)
+        with_outputs = step % 2 == 0
+        if with_outputs:
+            S.s3gd_step_ex(x, g, K, s.lr, ws, err=err, eta=eta, v=v, mu=mu or 0.0,
+                           opt_idx=idx if K else None, opt_signbits=sgn if K else None, opt_vote=vote)
+        else:
+            S.s3gd_step_ex(x, g, K, s.lr, ws, err=err, eta=eta, v=v, mu=mu or 0.0)
+        S.s3gd_device_status(ws)
+        xo_plain, e_o, idx_o, sgn_o, vote_o = O.error_feedback_step(x_o, g.cpu().numpy(), e_o, eta, K, s.lr,
+                                                                    topk=O.topk_sign_threshold)
+        if mu is None:
+            x_o = xo_plain
+        else:
+            x_o, v_o = O.apply_vote_momentum(x_o, v_o, vote_o, mu, s.lr)
+            assert np.array_equal(bits(v.cpu().numpy()), bits(v_o)), f"step {step}: momentum differs"
+        assert np.array_equal(bits(err.cpu().numpy()), bits(e_o)), f"step {step}: error memory differs"
+        assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)), f"step {step}: x differs"
+        if with_outputs:
+            assert np.array_equal(vote.cpu().numpy(), vote_o), f"step {step}: votes differ"
+            if K:
+                assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"step {step}: message differs"
+
+
+def test_step_ex_without_options_is_the_plain_step():
+    s = W.spec("resnet18", d=200_003, M=5)
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    ws = S.alloc_workspace(s.M, s.d, 2000, DEV)
+    xa, xb = x.clone(), x.clone()
+    S.s3gd_step(xa, g, 2000, s.lr, ws)
+    S.s3gd_step_ex(xb, g, 2000, s.lr, ws)
+    S.s3gd_device_status(ws)
+    assert torch.equal(xa, xb)
+
+
+def test_unfused_momentum_update():
+    d = 100_003
+    gen = torch.Generator(DEV).manual_seed(5)
+    x = torch.randn(d, device=DEV, generator=gen)
+    v = torch.randn(d, device=DEV, generator=gen)
+    vote = torch.randint(-1, 2, (d,), device=DEV, generator=gen, dtype=torch.int8)
+    x_o, v_o = O.apply_vote_momentum(x.cpu().numpy(), v.cpu().numpy(), vote.cpu().numpy(), 0.9, 1e-3)
+    S.s3gd_apply_momentum(x, v, vote, 0.9, 1e-3)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)) and np.array_equal(bits(v.cpu().numpy()), bits(v_o))
+
+
 def test_majority_vote_semantics_and_range_flag():
     d, M, K = 10, 2, 4
     idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)

@@ -69,6 +69,9 @@ def test_bad_arguments_rejected_before_launch(lib):
     assert lib.s3gd_step(fake, fake, 1, 8, 2, 0.1, fake, None, None, fake, 1 << 30, None) == INV  # idx without signs
     assert lib.s3gd_step(fake, fake, 1, 8, 2, 0.1, None, None, None, fake, 8, None) == WS
     assert lib.s3gd_device_status(None, None, None) == WS
+    assert lib.s3gd_step_ex(None, fake, None, 1.0, None, 0.0, 1, 8, 2, 0.1, None, None, None, fake, 1 << 30, None) == INV
+    assert lib.s3gd_step_ex(fake, fake, vp(256 * 1024 + 1), 1.0, None, 0.0, 1, 8, 2, 0.1, None, None, None, fake, 1 << 30, None) == INV
+    assert lib.s3gd_apply_momentum(fake, None, fake, 8, 0.5, 0.1, None) == INV
 
 
 def test_binding_refuses_cpu_tensors(lib):

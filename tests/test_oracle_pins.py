@@ -352,9 +352,87 @@ def test_support_statistics_match_closed_forms():
     assert abs(hist[2] - c["voter_count_pmf"][2]) < 1e-3
 
 
+# ------------------------------------ error compensation and momentum (Eq. (5)-(6), Section 4.7)
+def pin_error_feedback(orc):
+    """Small integer-valued inputs (every fp32 operation exact), checked by brute force in Python ints."""
+    rng = np.random.default_rng(11)
+    M, d, K, eta = 3, 12, 4, 2.0
+    x = np.zeros(d, dtype=np.float32)
+    e = np.zeros((M, d), dtype=np.float32)
+    sent_total = np.zeros((M, d), dtype=np.int64)        # sum over steps of TopK(g) (values)
+    grad_total = np.zeros((M, d), dtype=np.int64)        # sum over steps of eta^(steps since) ... only for eta = 1 below
+    for t in range(4):
+        gt = rng.integers(-9, 10, (M, d)).astype(np.float32)
+        g_int = gt.astype(np.int64) + int(eta) * e.astype(np.int64)          # Eq. (5) in exact arithmetic
+        x_new, e_new, idx, sgn, vote = orc.error_feedback_step(x, gt, e, eta, K, 1.0)
+        per_worker = []
+        for m in range(M):
+            kept, neg = brute_topk_sign(g_int[m].astype(np.float64), K)
+            per_worker.append((kept, neg))
+            assert idx[m].tolist() == kept
+            want_e = g_int[m].copy(); want_e[kept] = 0                        # Eq. (6): g - TopK(g)
+            assert e_new[m].astype(np.int64).tolist() == want_e.tolist()
+            assert np.all(f32_bits(e_new[m][kept]) == 0)                      # +0, not -0
+        assert vote.tolist() == brute_vote(per_worker, d)
+        assert np.array_equal(x_new, x - vote.astype(np.float32))
+        x, e = x_new, e_new
+    # eta = 0: no memory, the step is the plain step on g~ and e = g~ - TopK(g~)
+    gt = rng.standard_normal((M, d)).astype(np.float32)
+    junk = rng.standard_normal((M, d)).astype(np.float32)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    xa, ea, ia, sa, va = orc.error_feedback_step(x0, gt, junk, 0.0, K, 0.1)
+    kept_all = [brute_topk_sign(gt[m], K)[0] for m in range(M)]
+    assert [ia[m].tolist() for m in range(M)] == kept_all
+    for m in range(M):
+        off = np.ones(d, bool); off[kept_all[m]] = False
+        assert np.array_equal(f32_bits(ea[m][off]), f32_bits(gt[m][off])) and np.all(ea[m][~off] == 0)
+    # eta = 1 over several steps: what was sent plus what is remembered is everything that came in
+    e = np.zeros((M, d), dtype=np.float32)
+    for t in range(5):
+        gt = rng.integers(-20, 21, (M, d)).astype(np.float32)
+        g = gt + e
+        _, e_new, idx, _, _ = orc.error_feedback_step(x0, gt, e, 1.0, K, 0.1)
+        for m in range(M):
+            sent_total[m][idx[m]] += g[m][idx[m]].astype(np.int64)
+        grad_total += gt.astype(np.int64)
+        e = e_new
+    assert np.array_equal(sent_total + e.astype(np.int64), grad_total)
+
+
+def pin_momentum(orc):
+    from fractions import Fraction
+    d = 6
+    vote = np.array([1, -1, 0, 1, 0, -1], dtype=np.int8)
+    # mu = 0: v is the vote and x moves exactly as in Eq. (7)
+    x = np.array([0.5, -0.25, 3.0, 1e-3, -7.0, 0.1], dtype=np.float32)
+    xn, vn = orc.apply_vote_momentum(x, np.full(d, 9.0, np.float32), vote, 0.0, 0.125)
+    assert vn.tolist() == vote.astype(np.float32).tolist()
+    want = (x.astype(np.float64) - 0.125 * vote).astype(np.float32)
+    assert np.array_equal(xn, want)
+    # mu = 1/2, lr = 1/4, the same vote T times: every quantity is a short dyadic fraction, exact in fp32
+    x = np.zeros(d, dtype=np.float32); v = np.zeros(d, dtype=np.float32)
+    fx = [Fraction(0)] * d; fv = [Fraction(0)] * d
+    for t in range(8):
+        x, v = orc.apply_vote_momentum(x, v, vote, 0.5, 0.25)
+        fv = [Fraction(1, 2) * a + int(s) for a, s in zip(fv, vote)]
+        fx = [a - Fraction(1, 4) * b for a, b in zip(fx, fv)]
+        assert [Fraction(float(a)) for a in v] == fv and [Fraction(float(a)) for a in x] == fx
+    # rounding order: fl(mu*v) first, then + vote; fl(lr*v) first, then x - .
+    x1, v1 = orc.apply_vote_momentum(np.array([1.0], np.float32), np.array([0.1], np.float32),
+                                     np.array([1], np.int8), np.float32(0.3), np.float32(0.7))
+    mv = np.float32(np.float32(0.3) * np.float32(0.1))
+    vv = np.float32(mv + np.float32(1.0))
+    assert v1[0] == vv and x1[0] == np.float32(np.float32(1.0) - np.float32(np.float32(0.7) * vv))
+
+
+def test_error_feedback_and_momentum():
+    pin_error_feedback(O)
+    pin_momentum(O)
+
+
 # ------------------------------------------- the pins notice planted mistakes
 ALL_PINS = [pin_bruteforce, pin_example1, pin_gamma_one_is_signsgd_mv, pin_single_worker,
-            pin_invariants, pin_apply_bits, pin_vote_semantics]
+            pin_invariants, pin_apply_bits, pin_vote_semantics, pin_error_feedback, pin_momentum]
 
 
 def _mutants():
@@ -431,13 +509,43 @@ def _mutants():
     def apply_double(x, vote, lr):              # update computed in fp64 product then added twice-rounded
         return (x + np.float32(-1.0) * (np.float32(lr) * vote.astype(np.float32)) + np.float32(0.0)).astype(np.float32) * np.float32(1.0) + np.float32(0.0)
 
-    return [("topk_sign", higher_index_wins), ("topk_sign", signed_not_magnitude), ("topk_sign", smallest_k),
+    real_ef, real_mom = O.error_feedback_step, O.apply_vote_momentum
+
+    def ef_memory_of_raw_gradient(x, gt, e, eta, K, lr, topk=None):     # e <- g~ - TopK(g) instead of g - TopK(g)
+        xn, en, i, s, v = real_ef(x, gt, e, eta, K, lr, topk)
+        en2 = np.asarray(gt, dtype=np.float32).copy()
+        for m in range(en2.shape[0]):
+            en2[m][i[m].astype(np.int64)] = 0
+        return xn, en2, i, s, v
+
+    def ef_kept_entries_not_cleared(x, gt, e, eta, K, lr, topk=None):
+        xn, en, i, s, v = real_ef(x, gt, e, eta, K, lr, topk)
+        g = (np.asarray(gt, np.float32) + np.float32(eta) * np.asarray(e, np.float32)).astype(np.float32)
+        return xn, g, i, s, v
+
+    def ef_eta_on_gradient(x, gt, e, eta, K, lr, topk=None):            # g = eta * g~ + e
+        return real_ef(x, (np.float32(eta) * np.asarray(gt, np.float32)).astype(np.float32),
+                       (np.asarray(e, np.float32) / np.float32(eta if eta else 1)).astype(np.float32), eta, K, lr, topk)
+
+    def momentum_uses_old_v(x, v, vote, mu, lr):                        # x moved with v before its update
+        xn = (np.asarray(x, np.float32) - np.float32(lr) * np.asarray(v, np.float32)).astype(np.float32)
+        _, vn = real_mom(x, v, vote, mu, lr)
+        return xn, vn
+
+    def momentum_decays_the_vote(x, v, vote, mu, lr):                   # v <- mu * (v + vote)
+        vn = (np.float32(mu) * (np.asarray(v, np.float32) + np.asarray(vote).astype(np.float32))).astype(np.float32)
+        return (np.asarray(x, np.float32) - np.float32(lr) * vn).astype(np.float32), vn
+
+    extra = [("error_feedback_step", ef_memory_of_raw_gradient), ("error_feedback_step", ef_kept_entries_not_cleared),
+             ("error_feedback_step", ef_eta_on_gradient), ("apply_vote_momentum", momentum_uses_old_v),
+             ("apply_vote_momentum", momentum_decays_the_vote)]
+    return extra + [("topk_sign", higher_index_wins), ("topk_sign", signed_not_magnitude), ("topk_sign", smallest_k),
             ("topk_sign", inverted_sign_bits), ("topk_sign", msb_first), ("topk_sign", zero_votes_nothing),
             ("majority_vote", vote_tie_positive), ("majority_vote", vote_set_semantics),
             ("apply_vote", apply_plus), ("apply_vote", apply_double)]
 
 
-@pytest.mark.parametrize("which", range(10))
+@pytest.mark.parametrize("which", range(15))
 def test_pins_catch_planted_mistakes(which, monkeypatch):
     name, fn = _mutants()[which]
     monkeypatch.setattr(O, name, fn)
