@@ -229,6 +229,15 @@ def run_ours(args):
     x = W.make_x(spec, dev)
     ws = S.alloc_workspace(M, d, K, dev)
     stream = torch.cuda.current_stream(dev)
+    extended = args.error_feedback or args.momentum is not None
+    err = torch.zeros((M, d), dtype=torch.float32, device=dev) if args.error_feedback else None
+    vmom = torch.zeros(d, dtype=torch.float32, device=dev) if args.momentum is not None else None
+
+    def one_step():
+        if extended:
+            S.s3gd_step_ex(x, grads, K, spec.lr, ws, err=err, eta=1.0, v=vmom, mu=args.momentum or 0.0)
+        else:
+            S.s3gd_step(x, grads, K, spec.lr, ws)
 
     def barrier():
         torch.cuda.synchronize(dev)
@@ -237,7 +246,7 @@ def run_ours(args):
             torch.cuda.synchronize(dev)
 
     for _ in range(max(args.warmup, 3)):
-        S.s3gd_step(x, grads, K, spec.lr, ws)
+        one_step()
     code, info = S.s3gd_device_status(ws)
 
     # ---- timed region: device-resident inputs, phase events recorded by the library
@@ -247,7 +256,7 @@ def run_ours(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        S.s3gd_step(x, grads, K, spec.lr, ws)
+        one_step()
     e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -269,7 +278,7 @@ def run_ours(args):
         f0.record(stream)
         for _ in range(e2e_steps):
             grads.copy_(host_g, non_blocking=True)
-            S.s3gd_step(x, grads, K, spec.lr, ws)
+            one_step()
             host_x.copy_(x, non_blocking=True)
         f1.record(stream)
         barrier()
@@ -286,6 +295,12 @@ def run_ours(args):
         ms_step = ms_total / args.steps
         value = whole_job_value(world, M, d, args.steps, ms_total)
         b_grad, b_dense, b_min = byte_models(M, d, K)
+        if args.error_feedback:                  # + read and write of the error memory (fused ideal: 12 B per element)
+            b_dense += 8 * M * d
+            b_min += 8 * M * d
+        if args.momentum is not None:            # + read and write of v
+            b_dense += 8 * d
+            b_min += 8 * d
         peak, peak_kind = measured_peak()
         mean_phase = [sum(p[k] for p in phases) / max(len(phases), 1) for k in range(5)]
         dominant = max(range(5), key=lambda k: mean_phase[k])
@@ -316,6 +331,8 @@ def run_ours(args):
             "gpu_launches": launches,
             "device_info": {"rows_off_single_read_route": info[1], "max_candidates_per_row": info[4]},
         }
+        if extended:
+            line["config"]["variant"] = {"error_feedback_eta": 1.0 if args.error_feedback else None, "momentum_mu": args.momentum}
         if args.M or args.d:
             line["config"]["note"] = "reduced case of the named workload (not the headline configuration)"
         if e2e_ms is not None:
@@ -347,6 +364,9 @@ def main():
     ap.add_argument("--K", type=int, default=0, help="sparsity (default: the workload's first K)")
     ap.add_argument("--M", type=int, default=0, help="override the number of workers (smaller case of the same recipe)")
     ap.add_argument("--d", type=int, default=0, help="override the model size (smaller case of the same recipe)")
+    ap.add_argument("--error-feedback", action="store_true",
+                    help="time s3gd_step_ex with error memory (eta = 1, the paper's default) instead of s3gd_step")
+    ap.add_argument("--momentum", type=float, default=None, help="also use the momentum update with this mu")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-rows", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")

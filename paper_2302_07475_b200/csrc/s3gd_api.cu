@@ -171,12 +171,12 @@ namespace {
 // entries are zeroed (it is `sel` itself when error compensation is on).  v: momentum buffer or NULL.
 s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v, float mu, int M, uint64_t d,
                       uint64_t K, float lr, uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
-                      const Layout& L, void* ws, cudaStream_t st) {
+                      const Layout& L, void* ws, cudaStream_t st, bool mark_start = true) {
   char* base = static_cast<char*>(ws);
   int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
   if (K == 0 || K == d) {
     S3GD_TRY(cudaMemsetAsync(base + L.off_hdr, 0, kHdrWords * sizeof(uint32_t), st));
-    for (int ph = kPhaseStart; ph < kPhaseApplied; ++ph) prof_mark(ph, st);
+    for (int ph = mark_start ? kPhaseStart : kPhaseSampled; ph < kPhaseApplied; ++ph) prof_mark(ph, st);
     if (K == 0) {
       if (opt_vote) S3GD_TRY(cudaMemsetAsync(opt_vote, 0, (size_t)d, st));
       if (v) {                                 // no votes, but the momentum still decays and moves x
@@ -197,7 +197,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
     prof_mark(kPhaseApplied, st);
     return S3GD_OK;
   }
-  prof_mark(kPhaseStart, st);
+  if (mark_start) prof_mark(kPhaseStart, st);
   S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
   S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, st));
@@ -240,11 +240,12 @@ s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta
   if (s != S3GD_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float* sel = grads;
+  prof_mark(kPhaseStart, st);                  // the accumulation counts into the first phase
   if (opt_err != nullptr) {                    // g = g~ + eta * e, kept in the error memory
     S3GD_TRY(launch_ef_accumulate(opt_err, grads, eta, (uint64_t)M * d, st));
     sel = opt_err;
   }
-  return step_impl(x, sel, opt_err, opt_v, mu, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws, st);
+  return step_impl(x, sel, opt_err, opt_v, mu, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws, st, false);
 }
 
 s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
