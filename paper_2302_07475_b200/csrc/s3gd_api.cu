@@ -138,7 +138,7 @@ s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, ui
     return S3GD_OK;
   }
   S3GD_TRY(cudaMemsetAsync(out_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, nullptr, st));
+  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, nullptr, nullptr, 0.f, st));
 }
 
 s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
@@ -171,7 +171,8 @@ namespace {
 // entries are zeroed (it is `sel` itself when error compensation is on).  v: momentum buffer or NULL.
 s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v, float mu, int M, uint64_t d,
                       uint64_t K, float lr, uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
-                      const Layout& L, void* ws, cudaStream_t st, bool mark_start = true) {
+                      const Layout& L, void* ws, cudaStream_t st, bool mark_start = true,
+                      const float* ef_raw = nullptr, float eta = 0.f) {
   char* base = static_cast<char*>(ws);
   int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
   if (K == 0 || K == d) {
@@ -200,7 +201,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
   if (mark_start) prof_mark(kPhaseStart, st);
   S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, st));
+  S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, ef_raw, eta, st));
   cudaError_t e = v ? launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st)
                     : launch_counter_apply(counter, x, d, lr, opt_vote, st);
   prof_mark(kPhaseApplied, st);
@@ -241,11 +242,18 @@ s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float* sel = grads;
   prof_mark(kPhaseStart, st);                  // the accumulation counts into the first phase
+  const float* ef_raw = nullptr;
   if (opt_err != nullptr) {                    // g = g~ + eta * e, kept in the error memory
-    S3GD_TRY(launch_ef_accumulate(opt_err, grads, eta, (uint64_t)M * d, st));
+    // The filter pass can form g itself while it streams (one read of g~ and e, one write of g)
+    // when there is a filter pass and both buffers allow the same 16-byte accesses.
+    const bool fused = L.cap > 0 && K != 0 && K != d &&
+                       ((reinterpret_cast<uintptr_t>(opt_err) ^ reinterpret_cast<uintptr_t>(grads)) & 15u) == 0;
+    if (fused) ef_raw = grads;
+    else S3GD_TRY(launch_ef_accumulate(opt_err, grads, eta, (uint64_t)M * d, st));
     sel = opt_err;
   }
-  return step_impl(x, sel, opt_err, opt_v, mu, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws, st, false);
+  return step_impl(x, sel, opt_err, opt_v, mu, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws, st, false, ef_raw,
+                   eta);
 }
 
 s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,

@@ -131,7 +131,7 @@ cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t 
 cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     uint32_t* hdr, uint32_t* hist, cudaStream_t st);
+                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, cudaStream_t st);
 struct EmitOut {
   uint32_t* idx;        // [M x K] or NULL
   uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
@@ -145,7 +145,9 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, float* err_to_clear, cudaStream_t st);
+                          int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st);
+// (ef_raw != NULL: error compensation fused into the filter pass -- ef_raw are the raw gradients g~,
+//  `grads` is the error memory, which holds e on entry and g = g~ + eta * e after the filter pass)
 // err <- grads + eta * err, element-wise over n entries (Eq. (5))
 cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint64_t n, cudaStream_t st);
 // v <- mu * v + sgn(counter); x <- x - lr * v (momentum form of the update)

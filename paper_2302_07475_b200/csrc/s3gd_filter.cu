@@ -29,17 +29,22 @@ constexpr int kSampleUnroll = 8;
 
 // The kernel also resets the row's selection state, its radix histogram and (block 0) the
 // status words, so that no separate initialisation launch is needed on this route.
+// kEF: the row to sample is g = g~ + eta * e, formed on the fly from the gradients and the
+// error memory (which still holds e at this point).
+template <bool kEF>
 __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 RowState* __restrict__ rows, uint32_t n_sample,
                                                                 uint32_t stride, uint32_t j_rank, uint32_t K,
                                                                 uint32_t* __restrict__ hdr,
-                                                                uint32_t* __restrict__ hist) {
+                                                                uint32_t* __restrict__ hist,
+                                                                const float* __restrict__ err, float eta) {
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
   __shared__ uint32_t s_pick[2];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t row = blockIdx.x;
   const uint32_t* rowp = gbits + (uint64_t)row * d;
+  const float* errp = kEF ? err + (uint64_t)row * d : nullptr;
 
   if (blockIdx.x == 0 && tid < (uint32_t)kHdrWords) hdr[tid] = 0u;
   if (tid == 0) {
@@ -51,7 +56,10 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
   __syncthreads();
   if (stride == 0) {                              // short row: every entry is inspected
-    for (uint32_t e = tid; e < n_sample; e += 1024) atomicAdd(&s_hist[(rowp[e] & kAbsMask) >> 16], 1u);
+    for (uint32_t e = tid; e < n_sample; e += 1024) {
+      const uint32_t b = kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e];
+      atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u);
+    }
   } else {
     const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
     for (uint32_t c0 = warp; c0 < n_chunks; c0 += 32 * kSampleUnroll) {
@@ -62,6 +70,7 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
         if (c < n_chunks) {
           const uint64_t pos = (uint64_t)c * stride + (mix32(c) % (stride - (kChunk - 1))) + lane;
           v[u] = __ldg(rowp + pos);
+          if (kEF) v[u] = ef_value(v[u], __ldg(errp + pos), eta);
         }
       }
 #pragma unroll
@@ -141,10 +150,12 @@ constexpr int kWarpStage = 64;                 // survivors a warp can stage per
 // sign-less bit patterns for every input (denormals are not flushed in this build).
 __device__ __forceinline__ bool hit(uint32_t b, float tau) { return !(fabsf(__uint_as_float(b)) < tau); }
 
-__global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
-                                                                 RowState* __restrict__ rows,
-                                                                 uint2* __restrict__ cand, uint32_t cap,
-                                                                 uint2* __restrict__ seg, uint32_t n_tiles) {
+template <bool kEF>
+__global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_kernel(const uint32_t* __restrict__ gbits, int M,
+                                                                           uint64_t d, RowState* __restrict__ rows,
+                                                                           uint2* __restrict__ cand, uint32_t cap,
+                                                                           uint2* __restrict__ seg, uint32_t n_tiles,
+                                                                           float* __restrict__ err, float eta) {
   __shared__ uint2 s_stage[2][kWarpsPerTile][kWarpStage];
   __shared__ __align__(16) uint32_t s_wtot[3][kWarpsPerTile];   // survivors per warp of tile k in slot k % 3
   __shared__ uint32_t s_base[2];
@@ -172,6 +183,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t*
     const bool whole = (uint64_t)head + (uint64_t)(t + 1) * kTileElems <= d;
     Tile T;
     load_tile(T, rowp, d, head, t);
+    if (kEF) ef_materialise(T, err + (uint64_t)row * d, eta);
     uint32_t run = 0;                              // survivors of this warp so far (uniform in the warp)
     if (whole) {
       uint2* wl = s_stage[par][warp];
@@ -294,10 +306,11 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_kernel(const uint32_t*
 // is cheaper than a vote and four ballots per iteration; survivors are staged per CTA.
 constexpr int kStageCap = 512;                 // survivors staged per tile (8 bytes each, two buffers)
 
-__global__ void __launch_bounds__(kTileThreads, 4) filter_scan_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
+template <bool kEF>
+__global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
                                                               RowState* __restrict__ rows, uint2* __restrict__ cand,
                                                               uint32_t cap, uint2* __restrict__ seg,
-                                                              uint32_t n_tiles) {
+                                                              uint32_t n_tiles, float* __restrict__ err, float eta) {
   __shared__ uint2 s_stage[2][kStageCap];
   __shared__ uint32_t s_wtot[2][kWarpsPerTile + 1];
   __shared__ uint32_t s_base[2];
@@ -314,6 +327,7 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_scan_kernel(const uint
     const float tau = __uint_as_float(rows[row].tau_lo);
     Tile T;
     load_tile(T, rowp, d, head, t);
+    if (kEF) ef_materialise(T, err + (uint64_t)row * d, eta);
     uint32_t flags[kTileIters];
 #pragma unroll
     for (int it = 0; it < kTileIters; ++it)
@@ -392,24 +406,25 @@ __global__ void __launch_bounds__(kTileThreads, 4) filter_scan_kernel(const uint
 }  // namespace
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     uint32_t* hdr, uint32_t* hist, cudaStream_t st) {
+                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, cudaStream_t st) {
+  // ef_err != NULL: gbits are the raw gradients g~, ef_err holds e and leaves holding g = g~ + eta * e
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
-  cudaError_t e = cudaFuncSetAttribute(sample_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
+  auto sample = ef_err ? sample_threshold_kernel<true> : sample_threshold_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  sample_threshold_kernel<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
-                                                   (uint32_t)L.K, hdr, hist);
+  sample<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank, (uint32_t)L.K, hdr, hist,
+                                  ef_err, eta);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   prof_mark(kPhaseSampled, st);
   count_launch(2);
-  uint64_t n_work = (uint64_t)L.M * L.n_tiles;
-  uint64_t blocks = n_work < (uint64_t)kSMs * 8 ? n_work : (uint64_t)kSMs * 8;
-  if ((uint64_t)L.typical_cand * 250u > L.d)
-    filter_scan_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
-  else
-    filter_kernel<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles);
+  const uint64_t n_work = (uint64_t)L.M * L.n_tiles;
+  const uint64_t blocks = n_work < (uint64_t)kSMs * 8 ? n_work : (uint64_t)kSMs * 8;
+  const bool dense = (uint64_t)L.typical_cand * 250u > L.d;
+  auto filter = dense ? (ef_err ? filter_scan_kernel<true> : filter_scan_kernel<false>)
+                      : (ef_err ? filter_kernel<true> : filter_kernel<false>);
+  filter<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles, ef_err, eta);
   return cudaGetLastError();
 }
 

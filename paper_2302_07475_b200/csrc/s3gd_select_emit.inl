@@ -346,7 +346,7 @@ inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)
 }  // namespace
 
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, float* err_to_clear, cudaStream_t st) {
+                          int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st) {
   char* base = static_cast<char*>(ws);
   uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
   RowState* rows = reinterpret_cast<RowState*>(base + L.off_rows);
@@ -366,7 +366,9 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   } while (0)
 
   if (use_filter) {
-    cudaError_t e = launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, st);
+    cudaError_t e = ef_raw ? launch_sample_and_filter(reinterpret_cast<const uint32_t*>(ef_raw), L, rows, cand, seg,
+                                                      hdr, hist, err_to_clear, eta, st)
+                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, st);
     if (e != cudaSuccess) return e;
   } else {
     init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);

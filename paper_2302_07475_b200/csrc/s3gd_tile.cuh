@@ -71,6 +71,56 @@ __device__ __forceinline__ void load_tile(Tile& T, const uint32_t* __restrict__ 
   T.head_bits = T.head_valid ? ld_stream_u32(rowp + lane) : 0u;
 }
 
+// Error compensation fused into the streaming pass (Eq. (5)): the tile holds g~; it becomes
+// g = g~ + eta * e (product rounded, then sum rounded) and g is written to the error memory,
+// where the later passes and Eq. (6) find it.  errp is the row of the error memory; it must
+// be congruent to the gradient row modulo 16 bytes (the host checks) so that the same
+// 16-byte accesses apply.  Done in halves of four iterations to bound the registers.
+__device__ __forceinline__ uint32_t ef_value(uint32_t g_tilde_bits, float e, float eta) {
+  return __float_as_uint(__fadd_rn(__uint_as_float(g_tilde_bits), __fmul_rn(eta, e)));
+}
+
+__device__ __forceinline__ void ef_materialise(Tile& T, float* __restrict__ errp, float eta) {
+#pragma unroll
+  for (int half = 0; half < kTileIters; half += 4) {
+    float4 e[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int it = half + i;
+      if (T.valid[it] == 0xFu) {
+        e[i] = *reinterpret_cast<const float4*>(errp + T.first(it));
+      } else {
+        e[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (T.valid[it] & 1u) e[i].x = errp[T.first(it)];
+        if (T.valid[it] & 2u) e[i].y = errp[T.first(it) + 1];
+        if (T.valid[it] & 4u) e[i].z = errp[T.first(it) + 2];
+        if (T.valid[it] & 8u) e[i].w = errp[T.first(it) + 3];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int it = half + i;
+      T.bits[it][0] = ef_value(T.bits[it][0], e[i].x, eta);
+      T.bits[it][1] = ef_value(T.bits[it][1], e[i].y, eta);
+      T.bits[it][2] = ef_value(T.bits[it][2], e[i].z, eta);
+      T.bits[it][3] = ef_value(T.bits[it][3], e[i].w, eta);
+      if (T.valid[it] == 0xFu) {
+        *reinterpret_cast<uint4*>(errp + T.first(it)) =
+            make_uint4(T.bits[it][0], T.bits[it][1], T.bits[it][2], T.bits[it][3]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (T.valid[it] >> q & 1u) errp[T.first(it) + q] = __uint_as_float(T.bits[it][q]);
+      }
+    }
+  }
+  if (T.head_valid) {
+    const uint32_t lane = threadIdx.x & 31;
+    T.head_bits = ef_value(T.head_bits, errp[lane], eta);
+    errp[lane] = __uint_as_float(T.head_bits);
+  }
+}
+
 // Ranks of flagged entries in ascending-index order.
 // flags[it] (low 4 bits) and head_flag mark entries; after the call
 //   rank of (it, slot) = lane_excl(it) + popc(flags[it] & ((1u << slot) - 1))  + block offset of (warp, it)

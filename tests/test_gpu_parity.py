@@ -318,6 +318,22 @@ def test_error_memory_and_momentum_over_steps(K, eta, mu):
                 assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"step {step}: message differs"
 
 
+def test_error_memory_with_its_own_alignment():
+    """The error memory starts 4 bytes off the gradients' alignment: the step must not assume they match."""
+    s = W.spec("resnet18", d=150_001, M=4)
+    d, M, K = s.d, s.M, 600
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    big = torch.zeros(M * d + 4, device=DEV)
+    err = big[1:1 + M * d].view(M, d)
+    e0 = torch.randn((M, d), device=DEV, generator=torch.Generator(DEV).manual_seed(3))
+    err.copy_(e0)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    x_o, e_o, _, _, _ = O.error_feedback_step(x.cpu().numpy(), g.cpu().numpy(), e0.cpu().numpy(), 0.75, K, s.lr)
+    S.s3gd_step_ex(x, g, K, s.lr, ws, err=err, eta=0.75)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(bits(err.cpu().numpy()), bits(e_o)) and np.array_equal(bits(x.cpu().numpy()), bits(x_o))
+
+
 def test_step_ex_without_options_is_the_plain_step():
     s = W.spec("resnet18", d=200_003, M=5)
     g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
