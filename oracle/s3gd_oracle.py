@@ -26,7 +26,8 @@ Readings where the paper is silent (all listed in the design notes):
 * the update is one fp32 round-to-nearest operation: x - lr or x + lr.
 
 All integer results are exact, so GPU output must equal them bit for bit.
-Also here: error compensation (Eq. (5)-(6)) and the momentum update (Section 4.7).
+Also here: error compensation (Eq. (5)-(6)), the momentum update (Section 4.7) and the
+random-K variant (Section 3.4, Algorithm 2).
 
 Parity status: every function below is pinned by tests that do not call it to
 build their expectation (brute-force rank counting, the printed worked
@@ -179,6 +180,83 @@ def apply_vote_momentum(x, v, vote, mu, lr):
     v_new = ((mu32 * v).astype(np.float32) + np.asarray(vote).astype(np.float32)).astype(np.float32)
     x_new = (x - (lr32 * v_new).astype(np.float32)).astype(np.float32)
     return x_new, v_new
+
+
+# --------------------------------------------------------------------------
+# Random-K variant (Section 3.4, Algorithm 2): RandKSign keeps K coordinates chosen
+# uniformly at random instead of the K largest.  The paper names no generator; the
+# reading taken here: worker m at iteration t keeps the coordinates
+# pi(0), pi(1), ..., pi(K-1) of a keyed pseudo-random permutation pi of [0, d), in
+# that order (a K-subset without repetition; with the key shared, the indices
+# themselves would not even have to be transmitted).  pi is a 4-round balanced
+# Feistel network on 2h bits (2^(2h) >= d) with cycle walking into [0, d)
+# (Black & Rogaway, "Ciphers with arbitrary finite domains", 2002); its round
+# function is the 32-bit integer mixer "lowbias32" (C. Wellons, 2018):
+#   v ^= v >> 16; v *= 0x7feb352d; v ^= v >> 15; v *= 0x846ca68b; v ^= v >> 16.
+# Each side (this file, the CUDA kernels) implements these definitions on its own.
+# --------------------------------------------------------------------------
+
+def _lowbias32(v: np.ndarray) -> np.ndarray:
+    v = v.astype(np.uint64)
+    v ^= v >> np.uint64(16)
+    v = (v * np.uint64(0x7FEB352D)) & np.uint64(0xFFFFFFFF)
+    v ^= v >> np.uint64(15)
+    v = (v * np.uint64(0x846CA68B)) & np.uint64(0xFFFFFFFF)
+    v ^= v >> np.uint64(16)
+    return v
+
+
+def randk_round_keys(seed: int, worker: int, step: int) -> np.ndarray:
+    """Four 32-bit round keys of worker `worker` at iteration `step` under `seed`."""
+    keys = np.zeros(4, dtype=np.uint64)
+    base = (int(seed) & 0xFFFFFFFF) ^ ((int(worker) * 0x9E3779B9) & 0xFFFFFFFF) ^ ((int(step) * 0x85EBCA6B) & 0xFFFFFFFF)
+    for r in range(4):
+        keys[r] = _lowbias32(np.array([(base + (r + 1) * 0x9E3779B9) & 0xFFFFFFFF], dtype=np.uint64))[0]
+    return keys
+
+
+def randk_permutation(j: np.ndarray, d: int, keys: np.ndarray) -> np.ndarray:
+    """pi(j) for every entry of j (all < d): Feistel on 2h bits, walked until the value is below d."""
+    h = 1
+    while (1 << (2 * h)) < d:
+        h += 1
+    mask = np.uint64((1 << h) - 1)
+    v = np.asarray(j, dtype=np.uint64).copy()
+    todo = np.ones(v.shape, dtype=bool)
+    while todo.any():
+        left, right = v[todo] >> np.uint64(h), v[todo] & mask
+        for r in range(4):
+            f = _lowbias32(right ^ keys[r]) & mask
+            left, right = right, left ^ f
+        v[todo] = (left << np.uint64(h)) | right
+        todo &= v >= np.uint64(d)                  # cycle walking: outside [0, d) -> apply pi again
+    return v.astype(np.uint32)
+
+
+def randk_sign(grads: np.ndarray, K: int, seed: int, step: int):
+    """RandKSign of every worker (Algorithm 2, the "send" line) in transmitted form.
+
+    Returns (idx [M, K] uint32 in generation order pi(0..K-1), signbits [M, ceil(K/32)]);
+    sign bit j is the IEEE sign of the entry at idx[j].
+    """
+    bits = _as_bits(grads)
+    M, d = bits.shape
+    if not 0 <= K <= d:
+        raise ValueError("K must be in [0, d]")
+    idx = np.zeros((M, K), dtype=np.uint32)
+    sgn = np.zeros((M, (K + 31) // 32), dtype=np.uint32)
+    for m in range(M):
+        idx[m] = randk_permutation(np.arange(K, dtype=np.uint64), d, randk_round_keys(seed, m, step))
+        sgn[m] = _pack_sign_bits_fast((bits[m][idx[m].astype(np.int64)] >> np.uint32(31)).astype(bool))
+    return idx, sgn
+
+
+def randk_step(x: np.ndarray, grads: np.ndarray, K: int, lr, seed: int, step: int):
+    """One iteration of Algorithm 2: RandKSign, majority vote, update.  Returns (x_new, idx, signbits, vote)."""
+    M, d = grads.shape
+    idx, sgn = randk_sign(grads, K, seed, step)
+    vote, _ = majority_vote(idx, sgn, M, K, d)
+    return apply_vote(x, vote, lr), idx, sgn, vote
 
 
 # --------------------------------------------------------------------------

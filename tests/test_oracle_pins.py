@@ -430,9 +430,135 @@ def test_error_feedback_and_momentum():
     pin_momentum(O)
 
 
+
+# ------------------------------------------------ random-K variant (Section 3.4, Algorithm 2)
+def pin_randk_subset(orc):
+    """RandK keeps K distinct coordinates below d; K = d keeps every coordinate exactly once;
+    the sign bit j is the sign of the entry at the j-th kept index."""
+    rng = np.random.default_rng(5)
+    for d in (1, 2, 3, 5, 16, 17, 64, 100, 1000, 4097, 70_001):
+        for K in sorted({0, 1, d // 3, d - 1, d} - {-1}):
+            M = 3
+            g = rng.standard_normal((M, d)).astype(np.float32)
+            g[:, ::7] = np.float32(-0.0)
+            idx, sgn = orc.randk_sign(g, K, seed=d * 31 + K, step=K)
+            assert idx.shape == (M, K) and sgn.shape == (M, (K + 31) // 32)
+            for m in range(M):
+                row = idx[m].astype(np.int64).tolist()
+                assert all(0 <= n < d for n in row)
+                assert len(set(row)) == K                                  # without repetition
+                if K == d:
+                    assert sorted(row) == list(range(d))
+                assert unpack(sgn[m], K).tolist() == [int(f32_bits(g[m][n:n + 1])[0] >> 31) for n in row]
+                if K % 32:
+                    assert int(sgn[m][-1]) >> (K % 32) == 0                # unused bits are 0
+    # a prefix property the transmitted form relies on: the K kept coordinates are the first K of the K' > K ones
+    g = rng.standard_normal((2, 5000)).astype(np.float32)
+    i1, _ = orc.randk_sign(g, 100, seed=9, step=4)
+    i2, _ = orc.randk_sign(g, 700, seed=9, step=4)
+    assert np.array_equal(i1, i2[:, :100])
+
+
+def pin_randk_k_equals_d_is_signsgd_mv(orc):
+    """With K = d nothing is dropped: Algorithm 2 is signSGD with majority vote whatever the permutation."""
+    rng = np.random.default_rng(6)
+    M, d = 7, 333
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    x = rng.standard_normal(d).astype(np.float32)
+    xn, idx, sgn, vote = orc.randk_step(x, g, d, 0.25, seed=1, step=0)
+    total = np.where(np.signbit(g), -1, 1).sum(axis=0)
+    assert vote.tolist() == np.sign(total).astype(np.int8).tolist()
+    assert np.array_equal(xn, (x.astype(np.float64) - 0.25 * np.sign(total)).astype(np.float32))
+
+
+def pin_randk_uniform_and_independent(orc):
+    """Uniform K-subsets drawn independently per worker and per iteration: every coordinate is kept with
+    probability K/N, the number of workers keeping one coordinate is Binomial(M, K/N) (Lemma 3) and the
+    fraction nobody keeps is (1 - K/N)^M (Example 2)."""
+    with open(os.path.join(GOLD, "closed_forms.json")) as f:
+        cases = {(c["N"], c["K"], c["M"]): c for c in json.load(f)["cases"]}
+    # one big draw
+    N, K, M = 200000, 2000, 16
+    c = cases[(N, K, M)]
+    g = np.ones((M, N), dtype=np.float32)
+    idx, _ = orc.randk_sign(g, K, seed=77, step=3)
+    voters = np.zeros(N, dtype=np.int64)
+    for m in range(M):
+        voters[idx[m].astype(np.int64)] += 1
+    sd = np.sqrt(c["alpha"] * (1 - c["alpha"]) / N)
+    assert abs((voters == 0).mean() - c["p_empty"]) < 5 * sd
+    hist = np.bincount(voters, minlength=M + 1) / N
+    for k in (1, 2, 3):
+        p = c["voter_count_pmf"][k]
+        assert abs(hist[k] - p) < 5 * np.sqrt(p * (1 - p) / N) + 1e-6
+    # many iterations on a small model: per-coordinate inclusion frequency is K/N everywhere (chi-square)
+    N, K, M = 4096, 256, 8
+    c = cases[(N, K, M)]
+    g = np.ones((M, N), dtype=np.float32)
+    steps = 120
+    kept = np.zeros(N, dtype=np.int64)
+    empty = 0
+    first = np.zeros(N, dtype=np.int64)
+    for t in range(steps):
+        idx, _ = orc.randk_sign(g, K, seed=123, step=t)
+        voters = np.zeros(N, dtype=np.int64)
+        for m in range(M):
+            voters[idx[m].astype(np.int64)] += 1
+            first[int(idx[m][0])] += 1
+        kept += voters
+        empty += int((voters == 0).sum())
+    draws = steps * M
+    expect = draws * K / N                                          # 60 per coordinate
+    chi2 = float(((kept - expect) ** 2 / (expect * (1 - K / N))).sum())
+    assert abs(chi2 - (N - 1)) < 6 * np.sqrt(2 * (N - 1)), chi2     # chi-square with N-1 degrees of freedom
+    assert abs(empty / (steps * N) - c["p_empty"]) < 5 * np.sqrt(c["p_empty"] * (1 - c["p_empty"]) / (steps * N))
+    assert first.max() <= 8                                         # pi(0) is spread out, not stuck on a few values
+    # different workers, iterations and seeds give different subsets
+    a, _ = orc.randk_sign(g[:2], K, seed=1, step=0)
+    b, _ = orc.randk_sign(g[:2], K, seed=1, step=1)
+    c2, _ = orc.randk_sign(g[:2], K, seed=2, step=0)
+    sets = [set(a[0].tolist()), set(a[1].tolist()), set(b[0].tolist()), set(c2[0].tolist())]
+    for i in range(4):
+        for j in range(i + 1, 4):
+            assert len(sets[i] & sets[j]) < 60                       # expected overlap K^2/N = 16
+
+
+def test_randk_pins():
+    pin_randk_subset(O)
+    pin_randk_k_equals_d_is_signsgd_mv(O)
+    pin_randk_uniform_and_independent(O)
+
+
+def test_randk_mixer_known_answers():
+    """The 32-bit mixer and the Feistel network restated in Python integers, for a handful of inputs."""
+    def mix(v):
+        v ^= v >> 16; v = (v * 0x7FEB352D) & 0xFFFFFFFF
+        v ^= v >> 15; v = (v * 0x846CA68B) & 0xFFFFFFFF
+        return v ^ (v >> 16)
+    vals = [0, 1, 0xFFFFFFFF, 0x12345678, 0x80000000]
+    assert O._lowbias32(np.array(vals, dtype=np.uint64)).tolist() == [mix(v) for v in vals]
+    assert mix(0) == 0 and mix(1) != 1
+    seed, worker, step, d = 42, 3, 7, 1000
+    base = (seed ^ (worker * 0x9E3779B9) ^ (step * 0x85EBCA6B)) & 0xFFFFFFFF
+    keys = [mix((base + (r + 1) * 0x9E3779B9) & 0xFFFFFFFF) for r in range(4)]
+    assert O.randk_round_keys(seed, worker, step).tolist() == keys
+    h = 5                                                            # 2^10 >= 1000
+    def perm(v):
+        while True:
+            L, R = v >> h, v & 31
+            for r in range(4):
+                L, R = R, L ^ (mix(R ^ keys[r]) & 31)
+            v = (L << h) | R
+            if v < d:
+                return v
+    js = list(range(0, 1000, 37))
+    assert O.randk_permutation(np.array(js), d, np.array(keys, dtype=np.uint64)).tolist() == [perm(j) for j in js]
+
+
 # ------------------------------------------- the pins notice planted mistakes
 ALL_PINS = [pin_bruteforce, pin_example1, pin_gamma_one_is_signsgd_mv, pin_single_worker,
-            pin_invariants, pin_apply_bits, pin_vote_semantics, pin_error_feedback, pin_momentum]
+            pin_invariants, pin_apply_bits, pin_vote_semantics, pin_error_feedback, pin_momentum,
+            pin_randk_subset, pin_randk_k_equals_d_is_signsgd_mv, pin_randk_uniform_and_independent]
 
 
 def _mutants():
@@ -536,7 +662,27 @@ def _mutants():
         vn = (np.float32(mu) * (np.asarray(v, np.float32) + np.asarray(vote).astype(np.float32))).astype(np.float32)
         return (np.asarray(x, np.float32) - np.float32(lr) * vn).astype(np.float32), vn
 
-    extra = [("error_feedback_step", ef_memory_of_raw_gradient), ("error_feedback_step", ef_kept_entries_not_cleared),
+    real_perm, real_keys = O.randk_permutation, O.randk_round_keys
+
+    def randk_modulo_instead_of_walk(j, d, keys):                       # out-of-range values folded back: repeats
+        h = 1
+        while (1 << (2 * h)) < d:
+            h += 1
+        v = real_perm(j, 1 << (2 * h), keys)
+        return (v.astype(np.uint64) % np.uint64(d)).astype(np.uint32)
+
+    def randk_same_subset_for_every_worker(seed, worker, step):
+        return real_keys(seed, 0, step)
+
+    def randk_same_subset_every_iteration(seed, worker, step):
+        return real_keys(seed, worker, 0)
+
+    def randk_identity_rounds(j, d, keys):                              # no mixing: keeps the first K coordinates
+        return np.asarray(j).astype(np.uint32)
+
+    extra_randk = [("randk_permutation", randk_modulo_instead_of_walk), ("randk_round_keys", randk_same_subset_for_every_worker),
+                   ("randk_round_keys", randk_same_subset_every_iteration), ("randk_permutation", randk_identity_rounds)]
+    extra = extra_randk + [("error_feedback_step", ef_memory_of_raw_gradient), ("error_feedback_step", ef_kept_entries_not_cleared),
              ("error_feedback_step", ef_eta_on_gradient), ("apply_vote_momentum", momentum_uses_old_v),
              ("apply_vote_momentum", momentum_decays_the_vote)]
     return extra + [("topk_sign", higher_index_wins), ("topk_sign", signed_not_magnitude), ("topk_sign", smallest_k),
@@ -545,7 +691,7 @@ def _mutants():
             ("apply_vote", apply_plus), ("apply_vote", apply_double)]
 
 
-@pytest.mark.parametrize("which", range(15))
+@pytest.mark.parametrize("which", range(19))
 def test_pins_catch_planted_mistakes(which, monkeypatch):
     name, fn = _mutants()[which]
     monkeypatch.setattr(O, name, fn)
