@@ -135,7 +135,7 @@ def physical_gpu_index(local_rank: int) -> int:
 
 
 # --------------------------------------------------------------------------- CPU side
-def oracle_sample_time(spec, K, rows, reps=1):
+def oracle_sample_time(spec, K, rows, reps=1, randk=False):
     """Times the oracle's whole step on `rows` workers of the workload at full d (host cores)."""
     import torch
     from oracle import s3gd_oracle as O
@@ -146,7 +146,7 @@ def oracle_sample_time(spec, K, rows, reps=1):
     times = []
     for _ in range(reps):
         t0 = time.perf_counter()
-        x, _, _, _ = O.step(x, g, K, s.lr)
+        x, _, _, _ = O.randk_step(x, g, K, s.lr, 1, 0) if randk else O.step(x, g, K, s.lr)
         times.append(time.perf_counter() - t0)
     return times, rows * s.d, torch.get_num_threads()
 
@@ -233,8 +233,13 @@ def run_ours(args):
     err = torch.zeros((M, d), dtype=torch.float32, device=dev) if args.error_feedback else None
     vmom = torch.zeros(d, dtype=torch.float32, device=dev) if args.momentum is not None else None
 
+    step_no = [0]
+
     def one_step():
-        if extended:
+        if args.randk:
+            step_no[0] += 1
+            S.s3gd_step_randk(x, grads, K, spec.lr, 20230207, step_no[0], ws)
+        elif extended:
             S.s3gd_step_ex(x, grads, K, spec.lr, ws, err=err, eta=1.0, v=vmom, mu=args.momentum or 0.0)
         else:
             S.s3gd_step(x, grads, K, spec.lr, ws)
@@ -306,6 +311,12 @@ def run_ours(args):
         dominant = max(range(5), key=lambda k: mean_phase[k])
         kernel_name = "signplane_step_kernel" if K == d else "filter_kernel"
         dom_ms = mean_phase[4] if K == d else mean_phase[1]
+        if args.randk:
+            # random-K never streams the gradients: M*K gathers of one 32-byte sector each, M*K integer
+            # atomics on the counters, then the counter pass (4 B read per coordinate, x touched where voted)
+            kernel_name, dom_ms = "randk_kernel", mean_phase[3]
+            b_grad = M * K * (32 + 8)
+            b_dense = b_min = b_grad + 4 * d + 4 * d
         achieved = b_grad / (dom_ms * 1e-3) / 1e9 if dom_ms > 0 else None
         tr = NCU_TRAFFIC.get(f"{spec.name}:{K}")
         traffic = tr["bytes"] if tr and tr.get("digest") == kernel_digest() else None
@@ -331,6 +342,8 @@ def run_ours(args):
             "gpu_launches": launches,
             "device_info": {"rows_off_single_read_route": info[1], "max_candidates_per_row": info[4]},
         }
+        if args.randk:
+            line["config"]["variant"] = {"selection": "RandKSign (Section 3.4)"}
         if extended:
             line["config"]["variant"] = {"error_feedback_eta": 1.0 if args.error_feedback else None, "momentum_mu": args.momentum}
         if args.M or args.d:
@@ -343,7 +356,7 @@ def run_ours(args):
             line["e2e"] = {"value": None, "unit": UNIT, "error": e2e_err}
         if world == 1 and not args.no_cpu_baseline:
             rows = args.cpu_rows
-            t, elems, threads = oracle_sample_time(spec, K, rows)
+            t, elems, threads = oracle_sample_time(spec, K, rows, randk=args.randk)
             line["cpu_baseline"] = {"value": elems / t[0], "unit": UNIT, "cores": 1, "kind": "oracle",
                                     "sample": f"{rows} of {M} workers at full d={d}, K={K}, one step, {t[0]:.1f} s",
                                     "host_cores_available": os.cpu_count()}
@@ -367,6 +380,8 @@ def main():
     ap.add_argument("--error-feedback", action="store_true",
                     help="time s3gd_step_ex with error memory (eta = 1, the paper's default) instead of s3gd_step")
     ap.add_argument("--momentum", type=float, default=None, help="also use the momentum update with this mu")
+    ap.add_argument("--randk", action="store_true",
+                    help="time s3gd_step_randk (RandKSign, Section 3.4) instead of s3gd_step")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-rows", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -151,6 +151,34 @@ S3GD_API s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote,
                                          void* stream);
 
 /*
+ * Random-K variant (Section 3.4: RandKSign = sgn(RandK(g)); Algorithm 2 is Algorithm 1 with
+ * TopKSign replaced by it).  Worker m keeps K coordinates drawn uniformly without repetition,
+ * independently of the other workers and of earlier iterations.  The paper names no
+ * generator; this library's is deterministic in (seed, step, m):
+ *   key_r = mix(base + (r+1) * 0x9E3779B9),  base = seed ^ (m * 0x9E3779B9) ^ (step * 0x85EBCA6B)   (mod 2^32)
+ *   mix(v): v ^= v>>16; v *= 0x7FEB352D; v ^= v>>15; v *= 0x846CA68B; v ^= v>>16             (mod 2^32)
+ *   pi = 4 Feistel rounds on 2h bits, h minimal with 2^(2h) >= d:  (L, R) <- (R, L ^ (mix(R ^ key_r) & (2^h - 1))),
+ *        applied again while the value is >= d (cycle walking)
+ * and the kept coordinates are pi(0), ..., pi(K-1) IN THAT ORDER (not ascending): entry j of
+ * out_idx is pi(j) and sign bit j is the IEEE sign bit of that entry.  A receiver that knows
+ * (seed, step, m) can regenerate the indices, so only the sign words need to travel.
+ * s3gd_majority_vote accepts this message as it is.
+ *
+ *  s3gd_randk_sign   arguments as s3gd_topk_sign plus seed, step
+ *  s3gd_step_randk   arguments as s3gd_step plus seed, step; equals
+ *                    s3gd_randk_sign -> s3gd_majority_vote -> s3gd_apply
+ * K == 0 writes nothing; K == d keeps everything (the step is then signSGD with majority vote).
+ * No error compensation: Section 3.4 notes that random selection does not need it.
+ */
+S3GD_API s3gd_status s3gd_randk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t seed, uint32_t step,
+                                     uint32_t* out_idx, uint32_t* out_signbits,
+                                     void* ws, size_t ws_bytes, void* stream);
+S3GD_API s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr,
+                                     uint32_t seed, uint32_t step,
+                                     uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
+                                     void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Waits for `stream`, then reports what the kernels of earlier calls on this
  * workspace recorded: S3GD_OK, S3GD_ERR_INDEX_RANGE or S3GD_ERR_INTERNAL.
  * The record is cleared by the next s3gd_topk_sign / s3gd_majority_vote / s3gd_step.

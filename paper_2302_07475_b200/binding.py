@@ -24,7 +24,8 @@ STATUS_NAMES = {
 
 EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
            "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
-           "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum")
+           "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
+           "s3gd_randk_sign", "s3gd_step_randk")
 
 
 class S3gdError(RuntimeError):
@@ -75,6 +76,11 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
                                  u32p, u32p, vp, vp, sz, vp]
     lib.s3gd_apply_momentum.restype = ctypes.c_int
     lib.s3gd_apply_momentum.argtypes = [vp, vp, vp, u64, ctypes.c_float, ctypes.c_float, vp]
+    u32 = ctypes.c_uint32
+    lib.s3gd_randk_sign.restype = ctypes.c_int
+    lib.s3gd_randk_sign.argtypes = [vp, ctypes.c_int, u64, u64, u32, u32, u32p, u32p, vp, sz, vp]
+    lib.s3gd_step_randk.restype = ctypes.c_int
+    lib.s3gd_step_randk.argtypes = [vp, vp, ctypes.c_int, u64, u64, ctypes.c_float, u32, u32, u32p, u32p, vp, vp, sz, vp]
     if path is None:
         _lib = lib
     return lib
@@ -236,3 +242,30 @@ def s3gd_apply_momentum(x: torch.Tensor, v: torch.Tensor, vote: torch.Tensor, mu
     with torch.cuda.device(x.device):
         code = load().s3gd_apply_momentum(*args, _stream(x))
     _check("s3gd_apply_momentum", code)
+
+
+def s3gd_randk_sign(grads: torch.Tensor, K: int, seed: int, step: int, out_idx: torch.Tensor,
+                    out_signbits: torch.Tensor, ws: torch.Tensor) -> None:
+    """RandKSign: out_idx [M, K] = pi(0..K-1) per worker (generation order), out_signbits [M, ceil(K/32)]."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (g, M, d, K, seed & 0xFFFFFFFF, step & 0xFFFFFFFF, _ptr(out_idx, torch.int32, M * K, "out_idx"),
+            _ptr(out_signbits, torch.int32, M * words(K), "out_signbits"),
+            _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(grads.device):
+        code = load().s3gd_randk_sign(*args, _stream(grads))
+    _check("s3gd_randk_sign", code)
+
+
+def s3gd_step_randk(x: torch.Tensor, grads: torch.Tensor, K: int, lr: float, seed: int, step: int, ws: torch.Tensor,
+                    opt_idx: Optional[torch.Tensor] = None, opt_signbits: Optional[torch.Tensor] = None,
+                    opt_vote: Optional[torch.Tensor] = None) -> None:
+    """The fused step with RandKSign in place of TopKSign."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (_ptr(x, torch.float32, d, "x"), g, M, d, K, ctypes.c_float(lr), seed & 0xFFFFFFFF, step & 0xFFFFFFFF,
+            _ptr(opt_idx, torch.int32, M * K, "opt_idx"), _ptr(opt_signbits, torch.int32, M * words(K), "opt_signbits"),
+            _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(x.device):
+        code = load().s3gd_step_randk(*args, _stream(x))
+    _check("s3gd_step_randk", code)

@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libs3gd.so")
-SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu", "s3gd_select_small.cu", "s3gd_noalloc.cu"]
+SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu", "s3gd_select_small.cu", "s3gd_noalloc.cu", "s3gd_randk.cu"]
 HEADERS = ["s3gd_common.cuh", "s3gd_tile.cuh", "s3gd_select_emit.inl"]
 
 

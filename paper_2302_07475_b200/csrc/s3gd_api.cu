@@ -263,6 +263,44 @@ s3gd_status s3gd_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t
   return from_cuda(launch_apply_momentum(x, v, vote, d, mu, lr, static_cast<cudaStream_t>(stream)));
 }
 
+s3gd_status s3gd_randk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t seed, uint32_t step,
+                            uint32_t* out_idx, uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L) || grads == nullptr || !aligned(grads, 4)) return S3GD_ERR_INVALID_ARG;
+  if (K > 0 && (out_idx == nullptr || out_signbits == nullptr || !aligned(out_idx, 4) || !aligned(out_signbits, 4)))
+    return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* hdr = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + L.off_hdr);
+  S3GD_TRY(cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st));
+  return from_cuda(launch_randk(grads, M, d, K, seed, step, out_idx, out_signbits, nullptr, hdr, st));
+}
+
+s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t seed,
+                            uint32_t step, uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote, void* ws,
+                            size_t ws_bytes, void* stream) {
+  Layout L;
+  if (!make_layout(M, d, K, &L)) return S3GD_ERR_INVALID_ARG;
+  s3gd_status s = check_step_args(x, grads, opt_idx, opt_signbits);
+  if (s != S3GD_OK) return s;
+  s = check_ws(L, ws, ws_bytes);
+  if (s != S3GD_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(ws);
+  uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
+  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
+  prof_mark(kPhaseStart, st);
+  S3GD_TRY(cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st));
+  S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  for (int ph = kPhaseSampled; ph <= kPhaseThreshold; ++ph) prof_mark(ph, st);
+  S3GD_TRY(launch_randk(grads, M, d, K, seed, step, opt_idx, opt_signbits, counter, hdr, st));
+  prof_mark(kPhaseEmitted, st);
+  cudaError_t e = launch_counter_apply(counter, x, d, lr, opt_vote, st);
+  prof_mark(kPhaseApplied, st);
+  return from_cuda(e);
+}
+
 s3gd_status s3gd_profile_begin(int max_steps) {
   if (max_steps <= 0 || max_steps > (1 << 20) || g_prof.on) return S3GD_ERR_INVALID_ARG;
   const size_t n = (size_t)max_steps * kPhaseMarks;

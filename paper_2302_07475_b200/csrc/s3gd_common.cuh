@@ -157,5 +157,8 @@ cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64
                                   cudaStream_t st);
 // counter[n] <- sum over workers of (+1 | -1) by sign bit (K = d, when the sign counts are needed as such)
 cudaError_t launch_signplane_counts(const float* grads, int M, uint64_t d, int32_t* counter, cudaStream_t st);
+// RandKSign of every row under (seed, step): message if out_idx != NULL, votes added into counter if != NULL
+cudaError_t launch_randk(const float* grads, int M, uint64_t d, uint64_t K, uint32_t seed, uint32_t step,
+                         uint32_t* out_idx, uint32_t* out_signbits, int32_t* counter, uint32_t* hdr, cudaStream_t st);
 
 }  // namespace s3gd

@@ -357,6 +357,62 @@ def test_unfused_momentum_update():
     assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)) and np.array_equal(bits(v.cpu().numpy()), bits(v_o))
 
 
+# ------------------------------------------------ random-K variant (Section 3.4, Algorithm 2)
+def _randk_case(g, x, K, lr, seed, step, tag):
+    M, d = g.shape
+    gn, xn = g.cpu().numpy(), x.cpu().numpy()
+    x_o, idx_o, sgn_o, vote_o = O.randk_step(xn, gn, K, lr, seed, step)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    ws.fill_(0x5A)
+    idx = torch.full((M, max(K, 1)), -1, dtype=torch.int32, device=DEV)[:, :K].contiguous()
+    sgn = torch.full((M, max(S.binding.words(K), 1)), -1, dtype=torch.int32, device=DEV)[:, :S.binding.words(K)].contiguous()
+    vote = torch.full((d,), 77, dtype=torch.int8, device=DEV)
+    # message alone, then the library's own vote and update on it
+    S.s3gd_randk_sign(g, K, seed, step, idx, sgn, ws)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(u32(idx), idx_o), f"{tag}: indices differ"
+    assert np.array_equal(u32(sgn), sgn_o), f"{tag}: sign bits differ"
+    S.s3gd_majority_vote(idx, sgn, M, K, d, vote, ws)
+    xa = x.clone()
+    S.s3gd_apply(xa, vote, lr)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(vote.cpu().numpy(), vote_o), f"{tag}: votes differ"
+    assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"{tag}: unfused x differs"
+    # fused, with and without the optional outputs
+    idx.fill_(-1); sgn.fill_(-1); vote.fill_(77)
+    xb = x.clone()
+    S.s3gd_step_randk(xb, g, K, lr, seed, step, ws, idx, sgn, vote)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o) and np.array_equal(vote.cpu().numpy(), vote_o)
+    assert np.array_equal(bits(xb.cpu().numpy()), bits(x_o)), f"{tag}: fused x differs"
+    xc = x.clone()
+    S.s3gd_step_randk(xc, g, K, lr, seed, step, ws)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(bits(xc.cpu().numpy()), bits(x_o)), f"{tag}: fused (no outputs) x differs"
+
+
+@pytest.mark.parametrize("d,M,K", [(1, 1, 1), (2, 3, 1), (17, 4, 17), (1000, 3, 0), (4097, 5, 33), (65_536, 5, 655),
+                                   (65_537, 2, 65_537), (262_145, 7, 26_000), (1_199_882, 10, 12_000)])
+def test_randk_small_and_ragged(d, M, K):
+    s = W.spec("resnet18", d=d, M=M)
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    for step in (0, 3):
+        _randk_case(g, x, K, s.lr, seed=2023 + d, step=step, tag=f"randk d={d} K={K} step={step}")
+
+
+def test_randk_resnet18_full_size():
+    s = W.SPECS["resnet18"]
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    _randk_case(g, x, s.Ks[0], s.lr, seed=7, step=11, tag="randk resnet18")
+
+
+def test_randk_signed_zero_and_special_values():
+    d, M, K = 5000, 3, 2500
+    g = W.edge_case_grads("special", M, d, DEV)
+    x = torch.zeros(d, device=DEV)
+    _randk_case(g, x, K, 0.5, seed=1, step=1, tag="randk special")
+
+
 def test_majority_vote_semantics_and_range_flag():
     d, M, K = 10, 2, 4
     idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)

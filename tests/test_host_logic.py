@@ -72,6 +72,13 @@ def test_bad_arguments_rejected_before_launch(lib):
     assert lib.s3gd_step_ex(None, fake, None, 1.0, None, 0.0, 1, 8, 2, 0.1, None, None, None, fake, 1 << 30, None) == INV
     assert lib.s3gd_step_ex(fake, fake, vp(256 * 1024 + 1), 1.0, None, 0.0, 1, 8, 2, 0.1, None, None, None, fake, 1 << 30, None) == INV
     assert lib.s3gd_apply_momentum(fake, None, fake, 8, 0.5, 0.1, None) == INV
+    assert lib.s3gd_randk_sign(None, 1, 8, 2, 1, 0, fake, fake, fake, 1 << 30, None) == INV
+    assert lib.s3gd_randk_sign(fake, 1, 8, 9, 1, 0, fake, fake, fake, 1 << 30, None) == INV
+    assert lib.s3gd_randk_sign(fake, 1, 8, 2, 1, 0, fake, None, fake, 1 << 30, None) == INV
+    assert lib.s3gd_randk_sign(fake, 1, 8, 2, 1, 0, fake, fake, fake, 8, None) == WS
+    assert lib.s3gd_step_randk(None, fake, 1, 8, 2, 0.1, 1, 0, None, None, None, fake, 1 << 30, None) == INV
+    assert lib.s3gd_step_randk(fake, fake, 1, 8, 2, 0.1, 1, 0, fake, None, None, fake, 1 << 30, None) == INV
+    assert lib.s3gd_step_randk(fake, fake, 1, 8, 2, 0.1, 1, 0, None, None, None, None, 1 << 30, None) == WS
 
 
 def test_binding_refuses_cpu_tensors(lib):
