@@ -234,9 +234,18 @@ def run_ours(args):
     vmom = torch.zeros(d, dtype=torch.float32, device=dev) if args.momentum is not None else None
 
     step_no = [0]
+    if args.unfused:                            # the three calls with the message written to device memory
+        words = S.binding.words(K)
+        m_idx = torch.empty((M, K), dtype=torch.int32, device=dev)
+        m_sgn = torch.empty((M, words), dtype=torch.int32, device=dev)
+        m_vote = torch.empty(d, dtype=torch.int8, device=dev)
 
     def one_step():
-        if args.randk:
+        if args.unfused:
+            S.s3gd_topk_sign(grads, K, m_idx, m_sgn, ws)
+            S.s3gd_majority_vote(m_idx, m_sgn, M, K, d, m_vote, ws)
+            S.s3gd_apply(x, m_vote, spec.lr)
+        elif args.randk:
             step_no[0] += 1
             S.s3gd_step_randk(x, grads, K, spec.lr, 20230207, step_no[0], ws)
         elif extended:
@@ -344,6 +353,10 @@ def run_ours(args):
         }
         if args.randk:
             line["config"]["variant"] = {"selection": "RandKSign (Section 3.4)"}
+        if args.unfused:
+            line["config"]["variant"] = {"calls": "s3gd_topk_sign + s3gd_majority_vote + s3gd_apply"}
+            line["roofline"] = None             # the phase events belong to s3gd_step; only the step time is reported
+            line["phase_ms"] = None
         if extended:
             line["config"]["variant"] = {"error_feedback_eta": 1.0 if args.error_feedback else None, "momentum_mu": args.momentum}
         if args.M or args.d:
@@ -380,6 +393,8 @@ def main():
     ap.add_argument("--error-feedback", action="store_true",
                     help="time s3gd_step_ex with error memory (eta = 1, the paper's default) instead of s3gd_step")
     ap.add_argument("--momentum", type=float, default=None, help="also use the momentum update with this mu")
+    ap.add_argument("--unfused", action="store_true",
+                    help="time the three separate calls (message written out) instead of the fused step")
     ap.add_argument("--randk", action="store_true",
                     help="time s3gd_step_randk (RandKSign, Section 3.4) instead of s3gd_step")
     ap.add_argument("--e2e-steps", type=int, default=5)
