@@ -240,8 +240,15 @@ def run_ours(args):
         m_sgn = torch.empty((M, words), dtype=torch.int32, device=dev)
         m_vote = torch.empty(d, dtype=torch.int8, device=dev)
 
+    sharded = None
+    if args.shard_rows:                         # every rank's M rows are M of the job's world*M workers
+        from paper_2302_07475_b200.sharded import ShardedStep
+        sharded = ShardedStep(M, d, K, dev)
+
     def one_step():
-        if args.unfused:
+        if sharded is not None:
+            sharded.step(x, grads, spec.lr)
+        elif args.unfused:
             S.s3gd_topk_sign(grads, K, m_idx, m_sgn, ws)
             S.s3gd_majority_vote(m_idx, m_sgn, M, K, d, m_vote, ws)
             S.s3gd_apply(x, m_vote, spec.lr)
@@ -353,6 +360,12 @@ def run_ours(args):
         }
         if args.randk:
             line["config"]["variant"] = {"selection": "RandKSign (Section 3.4)"}
+        if sharded is not None:
+            line["config"]["parallelism"] = f"workers sharded over {world} rank(s), {world * M} workers in the vote"
+            line["config"]["variant"] = {"calls": "s3gd_topk_sign + all-gather of the message + s3gd_majority_vote + s3gd_apply",
+                                         "message_bytes_per_rank": sharded.message_bytes_per_rank()}
+            line["roofline"] = None
+            line["phase_ms"] = None
         if args.unfused:
             line["config"]["variant"] = {"calls": "s3gd_topk_sign + s3gd_majority_vote + s3gd_apply"}
             line["roofline"] = None             # the phase events belong to s3gd_step; only the step time is reported
@@ -393,6 +406,9 @@ def main():
     ap.add_argument("--error-feedback", action="store_true",
                     help="time s3gd_step_ex with error memory (eta = 1, the paper's default) instead of s3gd_step")
     ap.add_argument("--momentum", type=float, default=None, help="also use the momentum update with this mu")
+    ap.add_argument("--shard-rows", action="store_true",
+                    help="the deployment shape: each rank's rows are its own workers; the message is all-gathered "
+                         "and every rank votes over all of them (default: independent replicas)")
     ap.add_argument("--unfused", action="store_true",
                     help="time the three separate calls (message written out) instead of the fused step")
     ap.add_argument("--randk", action="store_true",
