@@ -43,7 +43,8 @@ __device__ __forceinline__ uint32_t block_scan_excl_1024(uint32_t v, uint32_t* s
 // kOrdered: the message (indices, sign bits) is wanted, so the candidates are laid out in index
 // order and emitted with their output positions.  Otherwise only the votes are wanted, whose
 // order does not matter: the candidates are copied as they lie, every entry above tau votes at
-// once, and only the entries equal to tau are ranked by index among themselves.
+// once, and only the entries equal to tau are ranked by index among themselves: pairwise up to
+// kMaxTiesUnordered of them, beyond that by a radix select on the index.
 constexpr uint32_t kMaxTiesUnordered = 1024;
 
 template <bool kOrdered>
@@ -191,8 +192,60 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   if (!kOrdered) {
     // ---- votes only.  Entries equal to tau are few as a rule; they are kept by ascending index
     // until `take` are taken, which needs their rank among themselves only.
-    const bool rank_ties = n_equal > take;                       // otherwise every one of them is kept
-    if (rank_ties && n_equal > kMaxTiesUnordered) return;        // too many to rank here: the general passes do this row
+    bool rank_ties = n_equal > take;                             // otherwise every one of them is kept
+    uint32_t idx_limit = 0xFFFFFFFFu;                            // entries equal to tau are kept up to this index
+    if (rank_ties && n_equal > kMaxTiesUnordered) {
+      // Too many to rank pairwise: a second radix select, on the index, finds the take-th smallest
+      // index among the entries equal to tau (indices are distinct, so exactly `take` lie at or below it).
+      uint32_t iprefix = 0, t_rem = take;
+#pragma unroll 1
+      for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const int prev_shift = pass == 1 ? 21 : 10;
+        const int nbins = pass == 2 ? 1024 : 2048;
+        const uint32_t mask = (uint32_t)(nbins - 1);
+        for (int b = tid; b < nbins; b += kSmallThreads) s_hist[b] = 0u;
+        __syncthreads();
+        for (uint32_t i = tid; i < n; i += kSmallThreads) {
+          if ((s_bits[i] & kAbsMask) != tau) continue;
+          const uint32_t idx = s_idx[i];
+          if (pass == 0 || (idx >> prev_shift) == iprefix) atomicAdd(&s_hist[(idx >> shift) & mask], 1u);
+        }
+        __syncthreads();
+        const int per = nbins / kSmallThreads;                   // 2 or 1 bins per thread, ascending
+        uint32_t cb[2] = {0u, 0u}, mine = 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+          if (i < per) { cb[i] = s_hist[(int)tid * per + i]; mine += cb[i]; }
+        uint32_t total;
+        const uint32_t below = block_scan_excl_1024(mine, s_warp, &total);
+        if (tid == 0) s_sel[0] = 0xFFFFFFFFu;
+        __syncthreads();
+        if (below < t_rem && below + mine >= t_rem) {            // exactly one thread
+          uint32_t a = below;
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            if (i < per) {
+              if (a + cb[i] >= t_rem) { s_sel[0] = (uint32_t)((int)tid * per + i); s_sel[1] = a; break; }
+              a += cb[i];
+            }
+          }
+        }
+        __syncthreads();
+        uint32_t digit = s_sel[0];
+        const uint32_t a = s_sel[1];
+        if (digit == 0xFFFFFFFFu) {                              // cannot happen: take <= n_equal
+          if (tid == 0) atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
+          digit = 0u;
+        } else {
+          t_rem -= a;
+        }
+        iprefix = (iprefix << (pass == 2 ? 10 : 11)) | digit;
+        __syncthreads();
+      }
+      idx_limit = iprefix;
+      rank_ties = false;                                         // decided by idx_limit instead
+    }
     uint32_t* s_tie_idx = s_hist;                                // the histogram is no longer needed
     uint32_t* s_tie_neg = s_hist + kMaxTiesUnordered;
     if (tid == 0) s_sel[0] = 0u;
@@ -200,11 +253,11 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
 #pragma unroll 4
     for (uint32_t i = tid; i < n; i += kSmallThreads) {
       const uint32_t bits = s_bits[i], key = bits & kAbsMask;
-      if (key > tau || (key == tau && !rank_ties)) {
+      if (key > tau || (key == tau && !rank_ties && s_idx[i] <= idx_limit)) {
         const uint32_t idx = s_idx[i];
         atomicAdd(o.counter + idx, (bits >> 31) ? -1 : 1);
         if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
-      } else if (key == tau) {
+      } else if (rank_ties && key == tau) {
         const uint32_t slot = atomicAdd(&s_sel[0], 1u);
         s_tie_idx[slot] = s_idx[i];
         s_tie_neg[slot] = bits >> 31;

@@ -254,12 +254,12 @@ def test_rows_that_leave_the_single_read_route():
     assert info[1] == M - 1
 
 
-@pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900)])
+@pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900), (5_000, 2_500), (1025, 1)])
 def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
     """Many entries exactly at the K-th magnitude, more than are taken: the lowest indices must win.
 
-    Sized so that the row's survivors fit the single-CTA selection; 600 ties are ranked there,
-    3000 are more than it ranks on chip and the row goes to the general passes instead.
+    Sized so that the row's survivors fit the single-CTA selection; 600 ties are ranked there
+    pairwise, 3000 by a radix select on the index (votes only) or by the general passes (message).
     """
     M, d, n_big = 3, 200_000, 1000
     g = torch.Generator("cpu").manual_seed(n_ties * 7 + take)
