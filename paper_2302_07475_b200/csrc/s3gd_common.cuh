@@ -35,6 +35,7 @@ enum HeaderWord : int {
   kHdrBadIndex = 2,      // out-of-range indices skipped by the vote scatter
   kHdrBadCount = 3,      // rows whose selection size != K
   kHdrMaxCand = 4,       // largest candidate count of a row
+  kHdrRowsDone = 8,      // rows finished by the single-CTA selection (words 5..7 are reported as 0)
   kHdrWords = 64
 };
 enum DeviceFlag : uint32_t { kFlagIndexRange = 1u, kFlagInternal = 2u };

@@ -11,6 +11,8 @@
 // works only if its source is the live one (row_uses_candidates), so the host never
 // has to look at device state.  The per-row follow-up of a pass (choosing the digit,
 // scanning the per-tile counts) is done by whichever block finishes that row last.
+#include <cooperative_groups.h>
+
 #include "s3gd_tile.cuh"
 
 namespace s3gd {
@@ -32,6 +34,26 @@ __global__ void init_kernel(uint32_t* __restrict__ hdr, RowState* __restrict__ r
     rows[m] = rs;
   }
   for (uint64_t i = tid; i < (uint64_t)M * kHistBins; i += nthr) hist[i] = 0u;
+}
+
+// A row's state.  kFromL2: in the single-launch form the passes are separated by grid-wide
+// barriers and the state is rewritten between them by other SMs, so the fields that change are
+// taken from L2; a launch of its own starts with a clean L1 and reads them the ordinary way,
+// which measured faster.
+template <bool kFromL2>
+__device__ __forceinline__ RowState load_row_state(const RowState* p) {
+  if (!kFromL2) return *p;
+  RowState rs = {};
+  rs.tau_lo = p->tau_lo;
+  rs.n_cand = p->n_cand;
+  rs.exact = p->exact;
+  rs.done = p->done;
+  rs.prefix = __ldcg(&p->prefix);
+  rs.k_rem = __ldcg(&p->k_rem);
+  rs.tau = __ldcg(&p->tau);
+  rs.take_ties = __ldcg(&p->take_ties);
+  rs.n_emitted = __ldcg(&p->n_emitted);
+  return rs;
 }
 
 // True in exactly one block per row: the one that arrives after all others of that row have
@@ -81,7 +103,7 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
   s_sum[tid] = mine;
   if (tid == 0) { s_sel[0] = 0xFFFFFFFFu; s_sel[1] = 0u; }
   __syncthreads();
-  const uint32_t k_rem = rows[row].k_rem;
+  const uint32_t k_rem = __ldcg(&rows[row].k_rem);
   uint32_t above = 0;                                // entries in bins owned by higher threads
   for (int t = kSelThreads - 1; t > (int)tid; --t) above += s_sum[t];
   if (above < k_rem && above + mine >= k_rem) {      // exactly one thread
@@ -99,7 +121,7 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
       atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
       digit = 0u; a = 0u;
     }
-    const uint32_t prefix = (rows[row].prefix << pass_bits(pass)) | digit;
+    const uint32_t prefix = (__ldcg(&rows[row].prefix) << pass_bits(pass)) | digit;
     rows[row].prefix = prefix;
     rows[row].k_rem = k_rem - a;
     if (pass == kNumPasses - 1) {
@@ -109,33 +131,34 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
   }
 }
 
-// grid (gx_c + gx_r, M): the first gx_c blocks of a row walk its candidates, the others its tiles.
-__global__ void __launch_bounds__(kSelThreads, 6) hist_pick_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                                uint32_t n_tiles, const uint2* __restrict__ cand,
-                                                                uint32_t cap, RowState* __restrict__ rows, uint32_t K,
-                                                                uint32_t* __restrict__ hist,
-                                                                uint32_t* __restrict__ hdr, int pass, uint32_t gx_c) {
+// One (virtual) block of a histogram pass.  A row has gx blocks: the first gx_c walk its
+// candidates, the others its tiles; bx is the block's number within the row.
+template <bool kFromL2>
+__device__ __forceinline__ void hist_pick_block(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
+                                                const uint2* __restrict__ cand, uint32_t cap,
+                                                RowState* __restrict__ rows, uint32_t K, uint32_t* __restrict__ hist,
+                                                uint32_t* __restrict__ hdr, int pass, uint32_t gx_c, uint32_t bx,
+                                                uint32_t row, uint32_t gx) {
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_sum[kSelThreads];
   __shared__ uint32_t s_sel[2];
   __shared__ uint32_t s_flag;
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
+  const RowState rs = load_row_state<kFromL2>(rows + row);
   if (rs.done) return;                               // finished by the single-CTA selection (all blocks of the row agree)
   const bool use_c = row_uses_candidates(rs, K, cap);
-  const bool is_c = blockIdx.x < gx_c;
+  const bool is_c = bx < gx_c;
   const int nbins = 1 << pass_bits(pass);
   const uint32_t mask = (uint32_t)(nbins - 1);
   uint32_t* g_hist = hist + (uint64_t)row * kHistBins;
   bool worked = false;
-  if (is_c && use_c && (uint64_t)blockIdx.x * kSelThreads * 4 < rs.n_cand) {
+  if (is_c && use_c && (uint64_t)bx * kSelThreads * 4 < rs.n_cand) {
     worked = true;
     for (int b = threadIdx.x; b < nbins; b += kSelThreads) s_hist[b] = 0u;
     __syncthreads();
     const uint2* c = cand + (uint64_t)row * cap;
     // four entries per thread and round, all four loads issued before the first is used
     const uint32_t n = rs.n_cand, step = gx_c * kSelThreads * 4;
-    for (uint32_t base = blockIdx.x * kSelThreads * 4; base < n; base += step) {
+    for (uint32_t base = bx * kSelThreads * 4; base < n; base += step) {
       uint32_t key[4];
       bool on[4];
 #pragma unroll
@@ -154,8 +177,8 @@ __global__ void __launch_bounds__(kSelThreads, 6) hist_pick_kernel(const uint32_
     __syncthreads();
     const uint32_t* rowp = gbits + (uint64_t)row * d;
     const uint32_t head = row_head(rowp, d);
-    const uint32_t gx_r = gridDim.x - gx_c;
-    for (uint32_t t = blockIdx.x - gx_c; t < n_tiles; t += gx_r) {
+    const uint32_t gx_r = gx - gx_c;
+    for (uint32_t t = bx - gx_c; t < n_tiles; t += gx_r) {
       Tile T;
       load_tile(T, rowp, d, head, t);
       if (t == 0 && threadIdx.x < 32) {
@@ -180,7 +203,7 @@ __global__ void __launch_bounds__(kSelThreads, 6) hist_pick_kernel(const uint32_
       if (c) atomicAdd(&g_hist[b], c);
     }
   }
-  if (last_block_of_row(&rows[row].ticket_hist, gridDim.x, &s_flag))
+  if (last_block_of_row(&rows[row].ticket_hist, gx, &s_flag))
     pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel);
 }
 

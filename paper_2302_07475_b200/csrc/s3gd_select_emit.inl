@@ -110,7 +110,7 @@ __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles
                                          uint32_t* s_warp) {
   constexpr int kPer = 8;                            // consecutive tiles per thread and round
   const uint32_t tid = threadIdx.x;
-  const uint32_t take = rows[row].take_ties;
+  const uint32_t take = __ldcg(&rows[row].take_ties);
   uint32_t carry_eq = 0, carry_out = 0;
   for (uint32_t base = 0; base < n_tiles; base += kSelThreads * kPer) {
     const uint32_t t0 = base + tid * kPer;
@@ -143,7 +143,7 @@ __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles
     carry_out += tot_sel;
   }
   if (tid == 0) {
-    const RowState rs = rows[row];
+    const RowState rs = load_row_state<true>(rows + row);
     rows[row].n_emitted = carry_out;
     if (carry_out != K) {
       atomicAdd(hdr + kHdrBadCount, 1u);
@@ -154,23 +154,22 @@ __device__ __forceinline__ void scan_row(uint2* __restrict__ c, uint32_t n_tiles
   }
 }
 
-// grid (gx_c + gx_r, M)
-__global__ void __launch_bounds__(kSelThreads, 6) count_scan_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                                 uint32_t n_tiles, const uint2* __restrict__ cand,
-                                                                 uint32_t cap, const uint2* __restrict__ seg,
-                                                                 RowState* __restrict__ rows, uint32_t K,
-                                                                 uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
-                                                                 uint32_t gx_c) {
+// One (virtual) block of the counting pass; the last block of a row scans the row's counts.
+template <bool kFromL2>
+__device__ __forceinline__ void count_scan_block(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
+                                                 const uint2* __restrict__ cand, uint32_t cap,
+                                                 const uint2* __restrict__ seg, RowState* __restrict__ rows,
+                                                 uint32_t K, uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
+                                                 uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx) {
   __shared__ uint32_t s_gt[kWarpsPerTile], s_eq[kWarpsPerTile], s_warp[kSelThreads / 32];
   __shared__ uint32_t s_flag;
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
+  const RowState rs = load_row_state<kFromL2>(rows + row);
   if (rs.done) return;
   const bool use_c = row_uses_candidates(rs, K, cap);
-  const bool is_c = blockIdx.x < gx_c;
-  if (is_c && use_c) count_cand(cand, cap, seg, n_tiles, rs, row, blockIdx.x, gx_c, cnt);
-  else if (!is_c && !use_c) count_row(gbits, d, n_tiles, rs, row, blockIdx.x - gx_c, gridDim.x - gx_c, cnt, s_gt, s_eq);
-  if (last_block_of_row(&rows[row].ticket_count, gridDim.x, &s_flag))
+  const bool is_c = bx < gx_c;
+  if (is_c && use_c) count_cand(cand, cap, seg, n_tiles, rs, row, bx, gx_c, cnt);
+  else if (!is_c && !use_c) count_row(gbits, d, n_tiles, rs, row, bx - gx_c, gx - gx_c, cnt, s_gt, s_eq);
+  if (last_block_of_row(&rows[row].ticket_count, gx, &s_flag))
     scan_row(cnt + (uint64_t)row * n_tiles, n_tiles, rows, row, K, cap, hdr, s_warp);
 }
 
@@ -324,21 +323,98 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
   }
 }
 
-// grid (gx_c + gx_r, M)
-__global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
-                                                           uint32_t n_tiles, const uint2* __restrict__ cand,
-                                                           uint32_t cap, const uint2* __restrict__ seg,
-                                                           const uint2* __restrict__ scan,
-                                                           const RowState* __restrict__ rows, EmitOut o,
-                                                           uint32_t gx_c) {
+// One (virtual) block of the emission.
+template <bool kFromL2>
+__device__ __forceinline__ void emit_block(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
+                                           const uint2* __restrict__ cand, uint32_t cap, const uint2* __restrict__ seg,
+                                           const uint2* __restrict__ scan, const RowState* __restrict__ rows,
+                                           const EmitOut& o, uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx) {
   __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
-  const uint32_t row = blockIdx.y;
-  const RowState rs = rows[row];
+  const RowState rs = load_row_state<kFromL2>(rows + row);
   if (rs.done) return;
   const bool use_c = row_uses_candidates(rs, o.K, cap);
-  const bool is_c = blockIdx.x < gx_c;
-  if (is_c && use_c) emit_cand(cand, cap, seg, scan, n_tiles, rs, row, blockIdx.x, gx_c, o);
-  else if (!is_c && !use_c) emit_row(gbits, d, n_tiles, scan, rs, row, blockIdx.x - gx_c, gridDim.x - gx_c, o, s_wtot);
+  const bool is_c = bx < gx_c;
+  if (is_c && use_c) emit_cand(cand, cap, seg, scan, n_tiles, rs, row, bx, gx_c, o);
+  else if (!is_c && !use_c) emit_row(gbits, d, n_tiles, scan, rs, row, bx - gx_c, gx - gx_c, o, s_wtot);
+}
+
+// The passes as launches of their own, grid (gx, M): used when the general passes carry the
+// selection of every row, where more resident blocks and per-pass register budgets pay.
+__global__ void __launch_bounds__(kSelThreads, 6) hist_pick_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                   uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                                   uint32_t cap, RowState* __restrict__ rows, uint32_t K,
+                                                                   uint32_t* __restrict__ hist,
+                                                                   uint32_t* __restrict__ hdr, int pass, uint32_t gx_c) {
+  hist_pick_block<false>(gbits, d, n_tiles, cand, cap, rows, K, hist, hdr, pass, gx_c, blockIdx.x, blockIdx.y, gridDim.x);
+}
+
+__global__ void __launch_bounds__(kSelThreads, 6) count_scan_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                                    uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                                    uint32_t cap, const uint2* __restrict__ seg,
+                                                                    RowState* __restrict__ rows, uint32_t K,
+                                                                    uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
+                                                                    uint32_t gx_c) {
+  count_scan_block<false>(gbits, d, n_tiles, cand, cap, seg, rows, K, cnt, hdr, gx_c, blockIdx.x, blockIdx.y, gridDim.x);
+}
+
+__global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
+                                                              uint32_t n_tiles, const uint2* __restrict__ cand,
+                                                              uint32_t cap, const uint2* __restrict__ seg,
+                                                              const uint2* __restrict__ scan,
+                                                              const RowState* __restrict__ rows, EmitOut o,
+                                                              uint32_t gx_c) {
+  emit_block<false>(gbits, d, n_tiles, cand, cap, seg, scan, rows, o, gx_c, blockIdx.x, blockIdx.y, gridDim.x);
+}
+
+// The same passes as ONE cooperative launch -- three histogram passes, the counting pass and the
+// emission, separated by grid-wide barriers -- for the case in which the single-CTA selection is
+// expected to finish every row.  The kernel then finds nothing to do and returns at once: a step
+// in which every row stays on the fast route pays for one empty launch, not five.  If rows are
+// left over, the resident blocks take the virtual blocks of each pass in turn; this is slower
+// per row than the separate launches (fewer blocks, one register budget for all passes) and is
+// only meant for the odd row.
+struct GeneralArgs {
+  const uint32_t* gbits;
+  uint64_t d;
+  uint32_t n_tiles;
+  const uint2* cand;
+  uint32_t cap;
+  const uint2* seg;
+  uint2* cnt;
+  RowState* rows;
+  uint32_t K;
+  uint32_t* hist;
+  uint32_t* hdr;
+  EmitOut o;
+  uint32_t M, gx_hist_c, gx_tile_c, gx_r;
+};
+
+__global__ void __launch_bounds__(kSelThreads, 4) general_passes_kernel(const GeneralArgs a) {
+  cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+  // written by the previous launch, read-only here: every block takes the same branch
+  if (__ldcg(a.hdr + kHdrRowsDone) == a.M) return;
+  {
+    const uint32_t gx = a.gx_hist_c + a.gx_r, nvb = gx * a.M;
+    for (int pass = 0; pass < kNumPasses; ++pass) {
+      for (uint32_t vb = blockIdx.x; vb < nvb; vb += gridDim.x) {
+        hist_pick_block<true>(a.gbits, a.d, a.n_tiles, a.cand, a.cap, a.rows, a.K, a.hist, a.hdr, pass, a.gx_hist_c,
+                        vb % gx, vb / gx, gx);
+        __syncthreads();
+      }
+      grid.sync();
+    }
+  }
+  const uint32_t gx = a.gx_tile_c + a.gx_r, nvb = gx * a.M;
+  for (uint32_t vb = blockIdx.x; vb < nvb; vb += gridDim.x) {
+    count_scan_block<true>(a.gbits, a.d, a.n_tiles, a.cand, a.cap, a.seg, a.rows, a.K, a.cnt, a.hdr, a.gx_tile_c, vb % gx,
+                     vb / gx, gx);
+    __syncthreads();
+  }
+  grid.sync();
+  for (uint32_t vb = blockIdx.x; vb < nvb; vb += gridDim.x) {
+    emit_block<true>(a.gbits, a.d, a.n_tiles, a.cand, a.cap, a.seg, a.cnt, a.rows, a.o, a.gx_tile_c, vb % gx, vb / gx, gx);
+    __syncthreads();
+  }
 }
 
 inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)(v < lo ? lo : (v > hi ? hi : v)); }
@@ -393,18 +469,44 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
-  for (int pass = 0; pass < kNumPasses; ++pass) {
-    hist_pick_kernel<<<dim3(gx_hist_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, rows, K,
-                                                                        hist, hdr, pass, gx_hist_c);
+  if (only_fallback && ef_raw == nullptr && err_to_clear == nullptr) {
+    // as many blocks as can be resident together, and no more than the largest pass has virtual blocks
+    static int blocks_per_sm = 0;
+    if (blocks_per_sm == 0) {
+      cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, general_passes_kernel, kSelThreads, 0);
+      if (e != cudaSuccess) return e;
+      if (blocks_per_sm < 1) return cudaErrorLaunchOutOfResources;
+    }
+    int n_sm = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return cudaErrorUnknown;
+    GeneralArgs ga;
+    ga.gbits = gbits; ga.d = L.d; ga.n_tiles = L.n_tiles; ga.cand = cand; ga.cap = L.cap; ga.seg = seg; ga.cnt = cnt;
+    ga.rows = rows; ga.K = K; ga.hist = hist; ga.hdr = hdr; ga.o = o; ga.M = (uint32_t)M;
+    ga.gx_hist_c = gx_hist_c; ga.gx_tile_c = gx_tile_c; ga.gx_r = gx_r;
+    const uint64_t most = (uint64_t)(gx_hist_c > gx_tile_c ? gx_hist_c : gx_tile_c) + gx_r;
+    const unsigned grid = clampu(most * (uint64_t)M, 1, (uint64_t)blocks_per_sm * (uint64_t)n_sm);
+    void* kargs[] = {&ga};
+    cudaError_t ce = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(general_passes_kernel), dim3(grid),
+                                                 dim3(kSelThreads), kargs, 0, st);
+    if (ce != cudaSuccess) return ce;
+    count_launch();
+    prof_mark(kPhaseThreshold, st);
+  } else {
+    for (int pass = 0; pass < kNumPasses; ++pass) {
+      hist_pick_kernel<<<dim3(gx_hist_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, rows, K,
+                                                                          hist, hdr, pass, gx_hist_c);
+      S3GD_CHECK_LAUNCH();
+    }
+    prof_mark(kPhaseThreshold, st);
+    count_scan_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows,
+                                                                         K, cnt, hdr, gx_tile_c);
+    S3GD_CHECK_LAUNCH();
+    emit_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
+                                                                   gx_tile_c);
     S3GD_CHECK_LAUNCH();
   }
-  prof_mark(kPhaseThreshold, st);
-  count_scan_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows,
-                                                                       K, cnt, hdr, gx_tile_c);
-  S3GD_CHECK_LAUNCH();
-  emit_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
-                                                                 gx_tile_c);
-  S3GD_CHECK_LAUNCH();
 #undef S3GD_CHECK_LAUNCH
   prof_mark(kPhaseEmitted, st);
   return cudaSuccess;

@@ -283,6 +283,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
       rows[row].take_ties = take;
       rows[row].n_emitted = n_kept;
       rows[row].done = 1u;
+      atomicAdd(hdr + kHdrRowsDone, 1u);
       if (n_kept != o.K) {
         atomicAdd(hdr + kHdrBadCount, 1u);
         atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
@@ -342,6 +343,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     rows[row].take_ties = take;
     rows[row].n_emitted = carry_out;
     rows[row].done = 1u;
+    atomicAdd(hdr + kHdrRowsDone, 1u);
     if (carry_out != o.K) {
       atomicAdd(hdr + kHdrBadCount, 1u);
       atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
