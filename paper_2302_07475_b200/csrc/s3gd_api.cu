@@ -199,7 +199,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
     return S3GD_OK;
   }
   if (mark_start) prof_mark(kPhaseStart, st);
-  S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  if (!select_clears_counter(L)) S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
   S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, ef_raw, eta, st));
   cudaError_t e = v ? launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st)

@@ -132,7 +132,9 @@ cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t 
 cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, cudaStream_t st);
+                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
+                                     cudaStream_t st);
+// (zero_counter != NULL: the d vote counters there, 16-byte aligned, are cleared by the sampling launch)
 struct EmitOut {
   uint32_t* idx;        // [M x K] or NULL
   uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
@@ -147,6 +149,8 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
                           int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st);
+// Does launch_select clear the counters it adds into (true), or must the caller do so first?
+bool select_clears_counter(const Layout& L);
 // (ef_raw != NULL: error compensation fused into the filter pass -- ef_raw are the raw gradients g~,
 //  `grads` is the error memory, which holds e on entry and g = g~ + eta * e after the filter pass)
 // err <- grads + eta * err, element-wise over n entries (Eq. (5))

@@ -31,17 +31,27 @@ constexpr int kSampleUnroll = 8;
 // status words, so that no separate initialisation launch is needed on this route.
 // kEF: the row to sample is g = g~ + eta * e, formed on the fly from the gradients and the
 // error memory (which still holds e at this point).
+// Blocks beyond the M sampling blocks clear the vote counters (if asked to): sampling is
+// latency-bound and leaves SMs idle, so the clearing costs no time of its own.
 template <bool kEF>
 __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 RowState* __restrict__ rows, uint32_t n_sample,
                                                                 uint32_t stride, uint32_t j_rank, uint32_t K,
                                                                 uint32_t* __restrict__ hdr,
                                                                 uint32_t* __restrict__ hist,
-                                                                const float* __restrict__ err, float eta) {
+                                                                const float* __restrict__ err, float eta, uint32_t M,
+                                                                int32_t* __restrict__ zero, uint64_t n_zero) {
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
   __shared__ uint32_t s_pick[2];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (blockIdx.x >= M) {                          // a clearing block; `zero` is 16-byte aligned
+    const uint64_t n4 = n_zero / 4, nthr = (uint64_t)(gridDim.x - M) * 1024;
+    uint4* z4 = reinterpret_cast<uint4*>(zero);
+    for (uint64_t i = (uint64_t)(blockIdx.x - M) * 1024 + tid; i < n4; i += nthr) z4[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (blockIdx.x == M && tid < (uint32_t)(n_zero - n4 * 4)) zero[n4 * 4 + tid] = 0;
+    return;
+  }
   const uint32_t row = blockIdx.x;
   const uint32_t* rowp = gbits + (uint64_t)row * d;
   const float* errp = kEF ? err + (uint64_t)row * d : nullptr;
@@ -406,15 +416,24 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
 }  // namespace
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
-                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, cudaStream_t st) {
+                                     uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
+                                     cudaStream_t st) {
   // ef_err != NULL: gbits are the raw gradients g~, ef_err holds e and leaves holding g = g~ + eta * e
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
   auto sample = ef_err ? sample_threshold_kernel<true> : sample_threshold_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  sample<<<L.M, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank, (uint32_t)L.K, hdr, hist,
-                                  ef_err, eta);
+  // clearing blocks: the SMs the M sampling blocks leave idle, and never fewer than 32
+  unsigned n_clear = 0;
+  if (zero_counter) {
+    const unsigned used = (unsigned)L.M % (unsigned)kSMs;
+    n_clear = (unsigned)kSMs - used;
+    if (n_clear < 32u) n_clear += (unsigned)kSMs;
+  }
+  sample<<<(unsigned)L.M + n_clear, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
+                                                      (uint32_t)L.K, hdr, hist, ef_err, eta, (uint32_t)L.M, zero_counter,
+                                                      L.d);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   prof_mark(kPhaseSampled, st);

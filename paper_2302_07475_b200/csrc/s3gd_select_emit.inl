@@ -421,6 +421,8 @@ inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)
 
 }  // namespace
 
+bool select_clears_counter(const Layout& L) { return L.cap > 0; }   // the sampling launch does it
+
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
                           int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st) {
   char* base = static_cast<char*>(ws);
@@ -443,8 +445,8 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
 
   if (use_filter) {
     cudaError_t e = ef_raw ? launch_sample_and_filter(reinterpret_cast<const uint32_t*>(ef_raw), L, rows, cand, seg,
-                                                      hdr, hist, err_to_clear, eta, st)
-                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, st);
+                                                      hdr, hist, err_to_clear, eta, counter, st)
+                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, st);
     if (e != cudaSuccess) return e;
   } else {
     init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
