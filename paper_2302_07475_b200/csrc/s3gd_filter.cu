@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t mix32(uint32_t v) {   // integer finaliser, 
 // no more) spread evenly over the row with a hashed offset inside each stride, then
 // tau_lo = lower edge of the highest bin b with (#sampled >= b) >= j_rank.
 constexpr int kChunk = 32;
-constexpr int kSampleUnroll = 8;
+constexpr int kSampleUnroll = 16;
 
 // The kernel also resets the row's selection state, its radix histogram and (block 0) the
 // status words, so that no separate initialisation launch is needed on this route.
@@ -78,7 +78,8 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
       for (int u = 0; u < kSampleUnroll; ++u) {
         const uint32_t c = c0 + 32 * u;
         if (c < n_chunks) {
-          const uint64_t pos = (uint64_t)c * stride + (mix32(c) % (stride - (kChunk - 1))) + lane;
+          // offset inside the stride: hash scaled into [0, stride - 31) by a multiply-high (no division)
+          const uint64_t pos = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk - 1)) + lane;
           v[u] = __ldg(rowp + pos);
           if (kEF) v[u] = ef_value(v[u], __ldg(errp + pos), eta);
         }
