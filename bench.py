@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/, keyed by workload, with the digest of the kernel sources they were taken
 # at.  Reported only while the sources are unchanged.
 NCU_TRAFFIC = {
-    # 361.70 MB read+written for 8 rows (profiles/filter_kernel_resnet18_M8.md), traffic proportional to rows
+    # 361.70 MB read+written for 8 rows (the ncu summary of the filter kernel under profiles/), traffic proportional to rows
     "resnet18:11174": {"bytes": int(361.70e6 * 100 / 8), "digest": "4176ff12e7dfe05c"},
 }
 KERNEL_SOURCES = ("s3gd_filter.cu", "s3gd_tile.cuh", "s3gd_common.cuh")
