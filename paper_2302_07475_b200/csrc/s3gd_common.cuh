@@ -145,6 +145,10 @@ struct EmitOut {
 };
 cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* cand, const uint2* seg, uint32_t* hdr,
                                 const EmitOut& o, cudaStream_t st);
+// Votes only, rows too large for one SM: a cluster of 2 or 4 CTAs per row (cluster_size_for; 0 = none fits)
+uint32_t cluster_size_for(uint32_t n_cand);
+cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* cand, uint32_t* hdr, const EmitOut& o,
+                                  uint32_t cluster, cudaStream_t st);
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,

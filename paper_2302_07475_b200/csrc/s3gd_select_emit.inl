@@ -458,15 +458,20 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
   o.err = err_to_clear; o.d = L.d;
   o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
-  if (use_filter) {                                  // rows whose candidates fit one SM are finished here
-    cudaError_t e = launch_select_small(L, rows, cand, seg, hdr, o, st);
+  // Rows whose candidates fit one SM are finished by one CTA each; if only the votes are wanted and a
+  // typical row needs the shared memory of up to four SMs, by a cluster of CTAs each.
+  const bool votes_only = counter != nullptr && out_idx == nullptr && out_signbits == nullptr;
+  const uint32_t cluster = (use_filter && votes_only && !fits_single_cta(L.typical_cand)) ? cluster_size_for(L.typical_cand) : 0u;
+  if (use_filter) {
+    cudaError_t e = cluster ? launch_select_cluster(L, rows, cand, hdr, o, cluster, st)
+                            : launch_select_small(L, rows, cand, seg, hdr, o, st);
     if (e != cudaSuccess) return e;
   }
   // Blocks per row (each block strides over its row's candidates or tiles).  If a row's
   // candidates are expected to fit the single-CTA selection, these launches only serve the
   // odd row that did not fit or fell back to the whole-row route, and normally exit at once:
   // keep them small.  Otherwise they carry the selection of all rows: about eight CTAs per SM.
-  const bool only_fallback = use_filter && fits_single_cta(L.typical_cand);
+  const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);
   const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * (only_fallback ? 4 : 8) + M - 1) / M);
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;

@@ -277,6 +277,25 @@ def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
     assert info[1] == 0                      # no row fell back to the whole-row route
 
 
+@pytest.mark.parametrize("n_ties,take", [(20_000, 10_000), (20_000, 19_999), (500, 499), (3_000, 3_000)])
+def test_ties_at_the_threshold_in_a_row_that_needs_a_cluster(n_ties, take):
+    """The same with so many survivors per row that the votes-only step selects with a cluster of CTAs."""
+    M, d, n_big = 3, 3_000_000, 30_000
+    g = torch.Generator("cpu").manual_seed(n_ties * 11 + take)
+    rows = []
+    for m in range(M):
+        v = (torch.rand(d, generator=g) * 0.9).float()
+        perm = torch.randperm(d, generator=g)
+        v[perm[:n_big]] = 5.0 + torch.rand(n_big, generator=g)
+        v[perm[n_big:n_big + n_ties]] = 2.0
+        sign = torch.where(torch.rand(d, generator=g) < 0.5, -1.0, 1.0)
+        rows.append(v * sign)
+    grads = torch.stack(rows).contiguous().to(DEV)
+    x = torch.zeros(d, device=DEV)
+    info = check_all(grads, x, n_big + take, 0.25, tag=f"cluster ties {n_ties}/{take}")
+    assert info[1] == 0 and info[4] > 27_136     # served from the candidates, more of them than one SM holds
+
+
 # ------------------------------------------- error compensation and momentum (s3gd_step_ex)
 @pytest.mark.parametrize("K,eta,mu", [(300, 1.0, None), (300, 0.5, 0.9), (75_002, 1.0, None), (300_007, 1.0, 0.5),
                                       (0, 1.0, 0.5), (3_000, 0.0, None)])
