@@ -461,7 +461,14 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   // Rows whose candidates fit one SM are finished by one CTA each; if only the votes are wanted and a
   // typical row needs the shared memory of up to four SMs, by a cluster of CTAs each.
   const bool votes_only = counter != nullptr && out_idx == nullptr && out_signbits == nullptr;
-  const uint32_t cluster = (use_filter && votes_only && !fits_single_cta(L.typical_cand)) ? cluster_size_for(L.typical_cand) : 0u;
+  // With error compensation the residuals pile up just below the threshold, so rows run above the
+  // sampling estimate: take the next larger on-chip form there.
+  const uint32_t expect = err_to_clear ? 2u * L.typical_cand : L.typical_cand;
+  uint32_t cluster = 0u;
+  if (use_filter && votes_only) {
+    if (!fits_single_cta(expect)) cluster = cluster_size_for(expect);
+    if (cluster == 0u && !fits_single_cta(L.typical_cand)) cluster = cluster_size_for(L.typical_cand);
+  }
   if (use_filter) {
     cudaError_t e = cluster ? launch_select_cluster(L, rows, cand, hdr, o, cluster, st)
                             : launch_select_small(L, rows, cand, seg, hdr, o, st);
@@ -476,7 +483,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
-  if (only_fallback && ef_raw == nullptr && err_to_clear == nullptr) {
+  if (only_fallback) {
     // as many blocks as can be resident together, and no more than the largest pass has virtual blocks
     static int blocks_per_sm = 0;
     if (blocks_per_sm == 0) {
