@@ -230,6 +230,10 @@ S3GD_API s3gd_status s3gd_majority_vote_noalloc(const uint32_t* idx, const uint3
  * profiling session at a time.  The events are created and destroyed by these two calls.
  */
 S3GD_API s3gd_status s3gd_profile_begin(int max_steps);
+/* The same, but only the two events around the filter pass are recorded ([1] is valid, the other
+ * durations are reported as 0): event records between kernels cost a few microseconds each, so this
+ * is the form to leave on while a step is being timed as a whole. */
+S3GD_API s3gd_status s3gd_profile_begin_filter(int max_steps);
 S3GD_API s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches);
 
 #ifdef __cplusplus

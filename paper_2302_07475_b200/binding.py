@@ -25,7 +25,7 @@ STATUS_NAMES = {
 EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
            "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
            "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
-           "s3gd_randk_sign", "s3gd_step_randk")
+           "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter")
 
 
 class S3gdError(RuntimeError):
@@ -76,6 +76,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
                                  u32p, u32p, vp, vp, sz, vp]
     lib.s3gd_apply_momentum.restype = ctypes.c_int
     lib.s3gd_apply_momentum.argtypes = [vp, vp, vp, u64, ctypes.c_float, ctypes.c_float, vp]
+    lib.s3gd_profile_begin_filter.restype = ctypes.c_int
+    lib.s3gd_profile_begin_filter.argtypes = [ctypes.c_int]
     u32 = ctypes.c_uint32
     lib.s3gd_randk_sign.restype = ctypes.c_int
     lib.s3gd_randk_sign.argtypes = [vp, ctypes.c_int, u64, u64, u32, u32, u32p, u32p, vp, sz, vp]
@@ -187,6 +189,11 @@ PHASES = ("sample", "filter", "threshold", "emit", "apply")
 
 def s3gd_profile_begin(max_steps: int) -> None:
     _check("s3gd_profile_begin", load().s3gd_profile_begin(int(max_steps)))
+
+
+def s3gd_profile_begin_filter(max_steps: int) -> None:
+    """As s3gd_profile_begin, but only the filter pass is bracketed by events (the other phases read 0)."""
+    _check("s3gd_profile_begin_filter", load().s3gd_profile_begin_filter(int(max_steps)))
 
 
 def s3gd_profile_end(max_steps: int):

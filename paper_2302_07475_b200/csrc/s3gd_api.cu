@@ -66,6 +66,7 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
 namespace {
 struct Profiler {
   bool on = false;
+  bool filter_only = false;           // record only the two marks around the filter pass
   int max_steps = 0, n_steps = 0;
   cudaEvent_t* ev = nullptr;          // kPhaseMarks events per recorded step
   unsigned long long launches = 0;
@@ -74,7 +75,8 @@ struct Profiler {
 
 void prof_mark(int phase, cudaStream_t st) {
   if (!g_prof.on || g_prof.n_steps >= g_prof.max_steps) return;
-  cudaEventRecord(g_prof.ev[(size_t)g_prof.n_steps * kPhaseMarks + phase], st);
+  if (!g_prof.filter_only || phase == kPhaseSampled || phase == kPhaseFiltered)
+    cudaEventRecord(g_prof.ev[(size_t)g_prof.n_steps * kPhaseMarks + phase], st);
   if (phase == kPhaseApplied) ++g_prof.n_steps;
 }
 
@@ -301,7 +303,15 @@ s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uin
   return from_cuda(e);
 }
 
-s3gd_status s3gd_profile_begin(int max_steps) {
+namespace {
+s3gd_status profile_begin(int max_steps, bool filter_only);
+}
+
+s3gd_status s3gd_profile_begin(int max_steps) { return profile_begin(max_steps, false); }
+s3gd_status s3gd_profile_begin_filter(int max_steps) { return profile_begin(max_steps, true); }
+
+namespace {
+s3gd_status profile_begin(int max_steps, bool filter_only) {
   if (max_steps <= 0 || max_steps > (1 << 20) || g_prof.on) return S3GD_ERR_INVALID_ARG;
   const size_t n = (size_t)max_steps * kPhaseMarks;
   g_prof.ev = new cudaEvent_t[n];
@@ -316,9 +326,11 @@ s3gd_status s3gd_profile_begin(int max_steps) {
   g_prof.max_steps = max_steps;
   g_prof.n_steps = 0;
   g_prof.launches = 0;
+  g_prof.filter_only = filter_only;
   g_prof.on = true;
   return S3GD_OK;
 }
+}  // namespace
 
 s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches) {
   if (!g_prof.on) return S3GD_ERR_INVALID_ARG;
@@ -327,6 +339,10 @@ s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches) {
   for (int s = 0; s < g_prof.n_steps && ret == S3GD_OK && out_ms != nullptr; ++s) {
     for (int ph = 0; ph + 1 < kPhaseMarks; ++ph) {
       float ms = 0.f;
+      if (g_prof.filter_only && ph != kPhaseSampled) {
+        out_ms[(size_t)s * (kPhaseMarks - 1) + ph] = 0.f;
+        continue;
+      }
       if (cudaEventElapsedTime(&ms, g_prof.ev[(size_t)s * kPhaseMarks + ph],
                                g_prof.ev[(size_t)s * kPhaseMarks + ph + 1]) != cudaSuccess)
         ret = S3GD_ERR_CUDA;

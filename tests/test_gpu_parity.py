@@ -432,6 +432,29 @@ def test_randk_signed_zero_and_special_values():
     _randk_case(g, x, K, 0.5, seed=1, step=1, tag="randk special")
 
 
+@pytest.mark.parametrize("d,M,K", [(300_007, 6, 300), (300_007, 6, 9_000), (65_536, 5, 65_536)])
+def test_step_replayed_from_a_cuda_graph(d, M, K):
+    """The step enqueues work only (no allocation, no synchronisation), so it can be captured once and replayed."""
+    s = W.spec("resnet18", d=d, M=M)
+    g, x0 = W.make_grads(s, DEV), W.make_x(s, DEV)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    x = x0.clone()
+    S.s3gd_step(x, g, K, s.lr, ws)                     # warm-up outside the capture (first-use attribute calls)
+    torch.cuda.synchronize()
+    x.copy_(x0)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        S.s3gd_step(x, g, K, s.lr, ws)
+    x.copy_(x0)
+    x_ref = x0.cpu().numpy()
+    for _ in range(3):
+        graph.replay()
+        x_ref, _, _, _ = O.step(x_ref, g.cpu().numpy(), K, s.lr)
+    torch.cuda.synchronize()
+    S.s3gd_device_status(ws)
+    assert np.array_equal(bits(x.cpu().numpy()), bits(x_ref))
+
+
 def test_majority_vote_semantics_and_range_flag():
     d, M, K = 10, 2, 4
     idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)
