@@ -361,6 +361,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
 // CTA adds up the C histograms through distributed shared memory and takes the same decision,
 // so nothing is broadcast.  Entries equal to tau, if not all of them are kept, are cut by a
 // second radix select on the index (the lowest indices win).  Every CTA then votes for its slice.
+template <uint32_t C>
 __global__ void __launch_bounds__(kSmallThreads, 1)
 select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand, uint32_t cap,
                       uint32_t* __restrict__ hdr, EmitOut o) {
@@ -370,7 +371,7 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_warp[kSmallWarps];
   __shared__ uint32_t s_sel[2];
-  const uint32_t C = cluster.num_blocks(), rank = cluster.block_rank();
+  const uint32_t rank = cluster.block_rank();             // the launch gives the cluster C CTAs
   const uint32_t row = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31;
   const RowState rs = rows[row];
   const uint32_t n = rs.n_cand;
@@ -389,10 +390,15 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
     s_bits[i] = e.x;
     s_idx[i] = e.y;
   }
-  // bin `b` summed over the cluster
+  // bin `b` summed over the cluster (C is a template argument so that the remote loads are all
+  // issued before the first one is used)
   auto combined = [&](uint32_t b) {
+    uint32_t part[C];
+#pragma unroll
+    for (uint32_t q = 0; q < C; ++q) part[q] = cluster.map_shared_rank(s_hist, q)[b];
     uint32_t v = 0;
-    for (uint32_t q = 0; q < C; ++q) v += cluster.map_shared_rank(s_hist, q)[b];
+#pragma unroll
+    for (uint32_t q = 0; q < C; ++q) v += part[q];
     return v;
   };
   // One radix pass over a 2048- or 1024-bin histogram that every CTA has filled for its slice:
@@ -554,8 +560,9 @@ uint32_t cluster_size_for(uint32_t n_cand) {
 
 cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* cand, uint32_t* hdr, const EmitOut& o,
                                   uint32_t cluster, cudaStream_t st) {
-  cudaError_t e = cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)kSmallSelectBytes);
+  auto kernel = cluster == 2u ? select_cluster_kernel<2> : (cluster == 4u ? select_cluster_kernel<4> : select_cluster_kernel<8>);
+  if (cluster != 2u && cluster != 4u && cluster != 8u) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
   if (e != cudaSuccess) return e;
   uint64_t need = (uint64_t)((L.cap + cluster - 1) / cluster) * 8u;
   if (need > kSmallSelectBytes) need = kSmallSelectBytes;
@@ -571,7 +578,7 @@ cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, select_cluster_kernel, rows, cand, L.cap, hdr, o);
+  e = cudaLaunchKernelEx(&cfg, kernel, rows, cand, L.cap, hdr, o);
   if (e == cudaSuccess) count_launch();
   return e;
 }
