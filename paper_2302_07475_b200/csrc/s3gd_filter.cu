@@ -367,13 +367,21 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
     }
     if (total <= (uint32_t)kStageCap) {
       if (head_flag) s_stage[par][R.head_rank] = make_uint2(T.head_bits, lane);
+      // a lane rarely holds more than one survivor among its four entries of an iteration: walk
+      // the set bits instead of testing all four slots
 #pragma unroll
       for (int it = 0; it < kTileIters; ++it) {
-        if (flags[it] == 0u) continue;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          if (flags[it] >> q & 1u)
-            s_stage[par][rank_of(R, flags, it, q)] = make_uint2(T.bits[it][q], (uint32_t)(T.first(it) + q));
+        uint32_t f = flags[it];
+        if (f == 0u) continue;
+        uint32_t pos = R.warp_off + R.it_off[it] + R.lane_excl[it];
+        const uint32_t first = (uint32_t)T.first(it);
+        do {
+          const uint32_t q = (uint32_t)__ffs((int)f) - 1u;
+          const uint32_t lo = (q & 1u) ? T.bits[it][1] : T.bits[it][0];
+          const uint32_t hi = (q & 1u) ? T.bits[it][3] : T.bits[it][2];
+          s_stage[par][pos++] = make_uint2((q & 2u) ? hi : lo, first + q);
+          f &= f - 1u;
+        } while (f);
       }
       if (tid == 0) pend_base = atomicAdd(&rows[row].n_cand, total);
       pend_n = total; pend_row = row; pend_t = t;
