@@ -140,7 +140,7 @@ s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, ui
     return S3GD_OK;
   }
   S3GD_TRY(cudaMemsetAsync(out_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, nullptr, nullptr, 0.f, st));
+  return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, false, nullptr, nullptr, 0.f, st));
 }
 
 s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
@@ -184,7 +184,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
       if (opt_vote) S3GD_TRY(cudaMemsetAsync(opt_vote, 0, (size_t)d, st));
       if (v) {                                 // no votes, but the momentum still decays and moves x
         S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
-        S3GD_TRY(launch_counter_apply_momentum(counter, x, v, d, mu, lr, nullptr, st));
+        S3GD_TRY(launch_counter_apply_momentum(counter, false, x, v, d, mu, lr, nullptr, st));
       }
       prof_mark(kPhaseApplied, st);
       return S3GD_OK;
@@ -192,7 +192,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
     if (opt_idx) S3GD_TRY(launch_signplane_message(sel, M, d, opt_idx, opt_signbits, st));
     if (v) {
       S3GD_TRY(launch_signplane_counts(sel, M, d, counter, st));
-      S3GD_TRY(launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st));
+      S3GD_TRY(launch_counter_apply_momentum(counter, false, x, v, d, mu, lr, opt_vote, st));
     } else {
       S3GD_TRY(launch_signplane_step(x, sel, M, d, lr, opt_vote, st));
     }
@@ -201,11 +201,16 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
     return S3GD_OK;
   }
   if (mark_start) prof_mark(kPhaseStart, st);
-  if (!select_clears_counter(L)) S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  // every worker votes at most once per coordinate here, so up to 127 workers fit byte counters
+  const bool packed = M <= kPackedMaxWorkers;
+  if (!select_clears_counter(L)) {
+    if (packed) S3GD_TRY(cudaMemsetAsync(counter, 0x80, (size_t)((d + 3) / 4) * 4, st));
+    else S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  }
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
-  S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, err_to_clear, ef_raw, eta, st));
-  cudaError_t e = v ? launch_counter_apply_momentum(counter, x, v, d, mu, lr, opt_vote, st)
-                    : launch_counter_apply(counter, x, d, lr, opt_vote, st);
+  S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, packed, err_to_clear, ef_raw, eta, st));
+  cudaError_t e = v ? launch_counter_apply_momentum(counter, packed, x, v, d, mu, lr, opt_vote, st)
+                    : launch_counter_apply(counter, packed, x, d, lr, opt_vote, st);
   prof_mark(kPhaseApplied, st);
   return from_cuda(e);
 }
@@ -276,7 +281,7 @@ s3gd_status s3gd_randk_sign(const float* grads, int M, uint64_t d, uint64_t K, u
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint32_t* hdr = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + L.off_hdr);
   S3GD_TRY(cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st));
-  return from_cuda(launch_randk(grads, M, d, K, seed, step, out_idx, out_signbits, nullptr, hdr, st));
+  return from_cuda(launch_randk(grads, M, d, K, seed, step, out_idx, out_signbits, nullptr, false, hdr, st));
 }
 
 s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t seed,
@@ -294,11 +299,13 @@ s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uin
   int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
   prof_mark(kPhaseStart, st);
   S3GD_TRY(cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st));
-  S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
+  const bool packed = M <= kPackedMaxWorkers;     // a permutation: one vote per worker and coordinate
+  if (packed) S3GD_TRY(cudaMemsetAsync(counter, 0x80, (size_t)((d + 3) / 4) * 4, st));
+  else S3GD_TRY(cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st));
   for (int ph = kPhaseSampled; ph <= kPhaseThreshold; ++ph) prof_mark(ph, st);
-  S3GD_TRY(launch_randk(grads, M, d, K, seed, step, opt_idx, opt_signbits, counter, hdr, st));
+  S3GD_TRY(launch_randk(grads, M, d, K, seed, step, opt_idx, opt_signbits, counter, packed, hdr, st));
   prof_mark(kPhaseEmitted, st);
-  cudaError_t e = launch_counter_apply(counter, x, d, lr, opt_vote, st);
+  cudaError_t e = launch_counter_apply(counter, packed, x, d, lr, opt_vote, st);
   prof_mark(kPhaseApplied, st);
   return from_cuda(e);
 }

@@ -112,6 +112,25 @@ __host__ __device__ __forceinline__ bool fits_single_cta(uint32_t n_cand) {
 }
 #endif
 
+// Vote counters.  Plain form: one int32 per coordinate.  Packed form (fused steps with at most
+// kPackedMaxWorkers workers, each of which votes at most once per coordinate): one byte per
+// coordinate holding 128 + (sum of votes), four coordinates per 32-bit word.  A vote adds or
+// subtracts 1 << (8 * slot) in the word; because every byte stays within [1, 255] no carry or
+// borrow ever crosses into a neighbour, so one 32-bit atomic serves.  A quarter of the bytes
+// means the counters of a 25M-coordinate model stay in L2 while the votes arrive at random.
+constexpr int kPackedMaxWorkers = 127;
+constexpr uint32_t kPackedZero = 0x80808080u;
+#ifdef __CUDACC__
+__device__ __forceinline__ void add_vote(int32_t* counter, uint32_t packed, uint32_t idx, uint32_t neg) {
+  if (packed) {
+    const uint32_t inc = 1u << ((idx & 3u) * 8u);
+    atomicAdd(reinterpret_cast<uint32_t*>(counter) + (idx >> 2), neg ? 0u - inc : inc);
+  } else {
+    atomicAdd(counter + idx, neg ? -1 : 1);
+  }
+}
+#endif
+
 // ------------------------------------------------------------------ profiling
 // Optional event marks at the phase boundaries of s3gd_step (see s3gd_profile_begin).
 enum Phase : int { kPhaseStart = 0, kPhaseSampled, kPhaseFiltered, kPhaseThreshold, kPhaseEmitted, kPhaseApplied,
@@ -125,7 +144,7 @@ cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cud
 cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
                                 int32_t* counter, uint32_t* hdr, cudaStream_t st);
 cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st);
-cudaError_t launch_counter_apply(const int32_t* counter, float* x, uint64_t d, float lr, int8_t* opt_vote,
+cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, uint64_t d, float lr, int8_t* opt_vote,
                                  cudaStream_t st);
 cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t d, float lr, int8_t* opt_vote,
                                   cudaStream_t st);
@@ -133,12 +152,13 @@ cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
                                      uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
-                                     cudaStream_t st);
+                                     bool packed, cudaStream_t st);
 // (zero_counter != NULL: the d vote counters there, 16-byte aligned, are cleared by the sampling launch)
 struct EmitOut {
   uint32_t* idx;        // [M x K] or NULL
   uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
   int32_t* counter;     // [d] or NULL
+  uint32_t packed;      // 1: the counters are bytes (see add_vote)
   float* err;           // [M x d] or NULL: error memory whose kept entries are set to zero (Eq. (6))
   uint64_t d;
   uint32_t K, words;
@@ -152,7 +172,8 @@ cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* 
 // Top-K selection of every row; writes the message if out_idx != NULL and adds the
 // votes into counter if counter != NULL.
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st);
+                          int32_t* counter, bool packed, float* err_to_clear, const float* ef_raw, float eta,
+                          cudaStream_t st);
 // Does launch_select clear the counters it adds into (true), or must the caller do so first?
 bool select_clears_counter(const Layout& L);
 // (ef_raw != NULL: error compensation fused into the filter pass -- ef_raw are the raw gradients g~,
@@ -160,14 +181,15 @@ bool select_clears_counter(const Layout& L);
 // err <- grads + eta * err, element-wise over n entries (Eq. (5))
 cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint64_t n, cudaStream_t st);
 // v <- mu * v + sgn(counter); x <- x - lr * v (momentum form of the update)
-cudaError_t launch_counter_apply_momentum(const int32_t* counter, float* x, float* v, uint64_t d, float mu, float lr,
-                                          int8_t* opt_vote, cudaStream_t st);
+cudaError_t launch_counter_apply_momentum(const int32_t* counter, bool packed, float* x, float* v, uint64_t d, float mu,
+                                          float lr, int8_t* opt_vote, cudaStream_t st);
 cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
                                   cudaStream_t st);
 // counter[n] <- sum over workers of (+1 | -1) by sign bit (K = d, when the sign counts are needed as such)
 cudaError_t launch_signplane_counts(const float* grads, int M, uint64_t d, int32_t* counter, cudaStream_t st);
 // RandKSign of every row under (seed, step): message if out_idx != NULL, votes added into counter if != NULL
 cudaError_t launch_randk(const float* grads, int M, uint64_t d, uint64_t K, uint32_t seed, uint32_t step,
-                         uint32_t* out_idx, uint32_t* out_signbits, int32_t* counter, uint32_t* hdr, cudaStream_t st);
+                         uint32_t* out_idx, uint32_t* out_signbits, int32_t* counter, bool packed, uint32_t* hdr,
+                         cudaStream_t st);
 
 }  // namespace s3gd

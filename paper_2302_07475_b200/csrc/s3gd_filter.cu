@@ -40,16 +40,18 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
                                                                 uint32_t* __restrict__ hdr,
                                                                 uint32_t* __restrict__ hist,
                                                                 const float* __restrict__ err, float eta, uint32_t M,
-                                                                int32_t* __restrict__ zero, uint64_t n_zero) {
+                                                                int32_t* __restrict__ zero, uint64_t n_zero,
+                                                                uint32_t zero_word) {
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
   __shared__ uint32_t s_pick[2];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (blockIdx.x >= M) {                          // a clearing block; `zero` is 16-byte aligned
+  if (blockIdx.x >= M) {                          // a clearing block; `zero` is 16-byte aligned, n_zero words
     const uint64_t n4 = n_zero / 4, nthr = (uint64_t)(gridDim.x - M) * 1024;
     uint4* z4 = reinterpret_cast<uint4*>(zero);
-    for (uint64_t i = (uint64_t)(blockIdx.x - M) * 1024 + tid; i < n4; i += nthr) z4[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (blockIdx.x == M && tid < (uint32_t)(n_zero - n4 * 4)) zero[n4 * 4 + tid] = 0;
+    for (uint64_t i = (uint64_t)(blockIdx.x - M) * 1024 + tid; i < n4; i += nthr)
+      z4[i] = make_uint4(zero_word, zero_word, zero_word, zero_word);
+    if (blockIdx.x == M && tid < (uint32_t)(n_zero - n4 * 4)) zero[n4 * 4 + tid] = (int32_t)zero_word;
     return;
   }
   const uint32_t row = blockIdx.x;
@@ -426,7 +428,7 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
                                      uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
-                                     cudaStream_t st) {
+                                     bool packed, cudaStream_t st) {
   // ef_err != NULL: gbits are the raw gradients g~, ef_err holds e and leaves holding g = g~ + eta * e
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
@@ -442,7 +444,7 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   }
   sample<<<(unsigned)L.M + n_clear, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
                                                       (uint32_t)L.K, hdr, hist, ef_err, eta, (uint32_t)L.M, zero_counter,
-                                                      L.d);
+                                                      packed ? (L.d + 3) / 4 : L.d, packed ? kPackedZero : 0u);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   prof_mark(kPhaseSampled, st);

@@ -52,7 +52,8 @@ __device__ __forceinline__ uint32_t permute(uint32_t j, uint32_t d, uint32_t h, 
 __global__ void __launch_bounds__(256) randk_kernel(const uint32_t* __restrict__ gbits, int M, uint32_t d, uint32_t K,
                                                     uint32_t h, uint32_t seed, uint32_t step,
                                                     uint32_t* __restrict__ out_idx, uint32_t* __restrict__ out_signbits,
-                                                    int32_t* __restrict__ counter, uint32_t* __restrict__ hdr) {
+                                                    int32_t* __restrict__ counter, uint32_t packed,
+                                                    uint32_t* __restrict__ hdr) {
   const uint32_t words = (K + 31u) / 32u;
   const uint64_t total = (uint64_t)words * (uint64_t)M;
   const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -70,7 +71,7 @@ __global__ void __launch_bounds__(256) randk_kernel(const uint32_t* __restrict__
       const uint32_t n = permute(j, d, h, key, &gave_up);
       neg = (__ldg(gbits + (uint64_t)m * d + n) >> 31) != 0u;
       if (out_idx) out_idx[(uint64_t)m * K + j] = n;
-      if (counter) atomicAdd(counter + n, neg ? -1 : 1);
+      if (counter) add_vote(counter, packed, n, neg ? 1u : 0u);
     }
     const uint32_t word = __ballot_sync(0xFFFFFFFFu, neg);
     if (out_signbits && lane == 0) out_signbits[w] = word;
@@ -81,7 +82,8 @@ __global__ void __launch_bounds__(256) randk_kernel(const uint32_t* __restrict__
 }  // namespace
 
 cudaError_t launch_randk(const float* grads, int M, uint64_t d, uint64_t K, uint32_t seed, uint32_t step,
-                         uint32_t* out_idx, uint32_t* out_signbits, int32_t* counter, uint32_t* hdr, cudaStream_t st) {
+                         uint32_t* out_idx, uint32_t* out_signbits, int32_t* counter, bool packed, uint32_t* hdr,
+                         cudaStream_t st) {
   if (K == 0) return cudaSuccess;
   uint32_t h = 1;
   while ((1ull << (2 * h)) < d) ++h;
@@ -90,7 +92,7 @@ cudaError_t launch_randk(const float* grads, int M, uint64_t d, uint64_t K, uint
   const uint64_t cap = (uint64_t)kSMs * 8;
   if (blocks > cap) blocks = cap;
   randk_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(grads), M, (uint32_t)d, (uint32_t)K,
-                                                 h, seed, step, out_idx, out_signbits, counter, hdr);
+                                                 h, seed, step, out_idx, out_signbits, counter, packed ? 1u : 0u, hdr);
   count_launch();
   return cudaGetLastError();
 }

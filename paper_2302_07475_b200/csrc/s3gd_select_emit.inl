@@ -214,7 +214,7 @@ __device__ __forceinline__ void emit_cand(const uint2* __restrict__ cand, uint32
         const uint32_t neg = e.x >> 31;
         if (sel && pos < o.K) {
           if (o.idx) o.idx[(uint64_t)row * o.K + pos] = e.y;
-          if (o.counter) atomicAdd(o.counter + e.y, neg ? -1 : 1);
+          if (o.counter) add_vote(o.counter, o.packed, e.y, neg);
           if (o.err) o.err[(uint64_t)row * o.d + e.y] = 0.f;
         }
         if (o.signbits && selb) {
@@ -281,7 +281,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
       const uint32_t neg = T.head_bits >> 31;
       if (pos < o.K) {
         if (o.idx) o.idx[(uint64_t)row * o.K + pos] = lane;
-        if (o.counter) atomicAdd(o.counter + lane, neg ? -1 : 1);
+        if (o.counter) add_vote(o.counter, o.packed, lane, neg);
         if (o.err) o.err[(uint64_t)row * o.d + lane] = 0.f;
         if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
       }
@@ -300,7 +300,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
             const uint32_t n = (uint32_t)(T.first(it) + q);
             const uint32_t neg = T.bits[it][q] >> 31;
             if (o.idx) o.idx[(uint64_t)row * o.K + pos] = n;
-            if (o.counter) atomicAdd(o.counter + n, neg ? -1 : 1);
+            if (o.counter) add_vote(o.counter, o.packed, n, neg);
             if (o.err) o.err[(uint64_t)row * o.d + n] = 0.f;
             const uint32_t rel = (pos >> 5) - (p0 >> 5);      // 0..4: at most 128 entries per warp-iteration
 #pragma unroll
@@ -424,7 +424,8 @@ inline unsigned clampu(uint64_t v, uint64_t lo, uint64_t hi) { return (unsigned)
 bool select_clears_counter(const Layout& L) { return L.cap > 0; }   // the sampling launch does it
 
 cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_t* out_idx, uint32_t* out_signbits,
-                          int32_t* counter, float* err_to_clear, const float* ef_raw, float eta, cudaStream_t st) {
+                          int32_t* counter, bool packed, float* err_to_clear, const float* ef_raw, float eta,
+                          cudaStream_t st) {
   char* base = static_cast<char*>(ws);
   uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
   RowState* rows = reinterpret_cast<RowState*>(base + L.off_rows);
@@ -445,8 +446,8 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
 
   if (use_filter) {
     cudaError_t e = ef_raw ? launch_sample_and_filter(reinterpret_cast<const uint32_t*>(ef_raw), L, rows, cand, seg,
-                                                      hdr, hist, err_to_clear, eta, counter, st)
-                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, st);
+                                                      hdr, hist, err_to_clear, eta, counter, packed, st)
+                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, packed, st);
     if (e != cudaSuccess) return e;
   } else {
     init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
@@ -455,7 +456,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   }
   prof_mark(kPhaseFiltered, st);
   EmitOut o;
-  o.idx = out_idx; o.signbits = out_signbits; o.counter = counter;
+  o.idx = out_idx; o.signbits = out_signbits; o.counter = counter; o.packed = packed ? 1u : 0u;
   o.err = err_to_clear; o.d = L.d;
   o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
   // Rows whose candidates fit one SM are finished by one CTA each; if only the votes are wanted and a

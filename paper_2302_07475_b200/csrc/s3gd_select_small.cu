@@ -257,7 +257,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
       const uint32_t bits = s_bits[i], key = bits & kAbsMask;
       if (key > tau || (key == tau && !rank_ties && s_idx[i] <= idx_limit)) {
         const uint32_t idx = s_idx[i];
-        atomicAdd(o.counter + idx, (bits >> 31) ? -1 : 1);
+        add_vote(o.counter, o.packed, idx, bits >> 31);
         if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
       } else if (rank_ties && key == tau) {
         const uint32_t slot = atomicAdd(&s_sel[0], 1u);
@@ -274,7 +274,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
         uint32_t before = 0;
         for (uint32_t j = 0; j < e; ++j) before += (uint32_t)(s_tie_idx[j] < mine);
         if (before < take) {
-          atomicAdd(o.counter + mine, s_tie_neg[tid] ? -1 : 1);
+          add_vote(o.counter, o.packed, mine, s_tie_neg[tid]);
           if (o.err) o.err[(uint64_t)row * o.d + mine] = 0.f;
         }
       }
@@ -330,7 +330,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
           const uint32_t idx = s_idx[i0 + q];
           const uint32_t neg = bits[q] >> 31;
           if (o.idx) o.idx[(uint64_t)row * o.K + pos] = idx;
-          if (o.counter) atomicAdd(o.counter + idx, neg ? -1 : 1);
+          if (o.counter) add_vote(o.counter, o.packed, idx, neg);
           if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
           // sign bits only when the message is asked for: one atomic per negative entry
           if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
@@ -515,7 +515,7 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
     const uint32_t bits = s_bits[i], key = bits & kAbsMask;
     if (key > tau || (key == tau && s_idx[i] <= idx_limit)) {
       const uint32_t idx = s_idx[i];
-      atomicAdd(o.counter + idx, (bits >> 31) ? -1 : 1);
+      add_vote(o.counter, o.packed, idx, bits >> 31);
       if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
     }
   }

@@ -118,6 +118,48 @@ __global__ void __launch_bounds__(256) counter_apply_kernel(const int32_t* __res
   }
 }
 
+// The same for packed counters (one byte per coordinate holding 128 + count): a thread takes one
+// 32-bit word = four coordinates.  kVec: x is 16-byte aligned and opt_vote (if given) 4-byte aligned.
+template <bool kVec>
+__global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_t* __restrict__ cw,
+                                                                   float* __restrict__ x, uint64_t d, float lr,
+                                                                   int8_t* __restrict__ opt_vote) {
+  const uint64_t n_words = (d + 3) / 4;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride) {
+    const uint32_t w = cw[i];
+    if (w == kPackedZero && opt_vote == nullptr) continue;
+    int c[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) c[q] = (int)((w >> (8 * q)) & 0xFFu) - 128;
+    const bool full = i * 4 + 4 <= d;
+    if (kVec && full) {
+      if (opt_vote) {
+        uint32_t pk = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) pk |= (uint32_t)(uint8_t)(int8_t)((c[q] > 0) - (c[q] < 0)) << (8 * q);
+        *reinterpret_cast<uint32_t*>(opt_vote + i * 4) = pk;
+      }
+      if (w == kPackedZero) continue;
+      float4* px = reinterpret_cast<float4*>(x + i * 4);
+      float4 xv = *px;
+      if (c[0]) xv.x = moved(xv.x, c[0], lr);
+      if (c[1]) xv.y = moved(xv.y, c[1], lr);
+      if (c[2]) xv.z = moved(xv.z, c[2], lr);
+      if (c[3]) xv.w = moved(xv.w, c[3], lr);
+      *px = xv;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t n = i * 4 + q;
+        if (n >= d) break;
+        if (opt_vote) opt_vote[n] = (int8_t)((c[q] > 0) - (c[q] < 0));
+        if (c[q]) x[n] = moved(x[n], c[q], lr);
+      }
+    }
+  }
+}
+
 // err <- grads + eta * err: one rounding for the product, one for the sum (Eq. (5))
 __global__ void __launch_bounds__(256) ef_accumulate_kernel(float* __restrict__ err, const float* __restrict__ grads,
                                                             float eta, uint64_t n) {
@@ -146,13 +188,14 @@ __device__ __forceinline__ void momentum_update(float& x, float& v, int s, float
   x = __fsub_rn(x, __fmul_rn(lr, v));
 }
 
+template <bool kPacked>
 __global__ void __launch_bounds__(256) counter_apply_momentum_kernel(const int32_t* __restrict__ counter,
                                                                      float* __restrict__ x, float* __restrict__ v,
                                                                      uint64_t d, float mu, float lr,
                                                                      int8_t* __restrict__ opt_vote) {
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   for (uint64_t n = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; n < d; n += stride) {
-    const int c = counter[n];
+    const int c = kPacked ? (int)reinterpret_cast<const uint8_t*>(counter)[n] - 128 : counter[n];
     if (opt_vote) opt_vote[n] = (int8_t)((c > 0) - (c < 0));
     float xv = x[n], vv = v[n];
     momentum_update(xv, vv, c, mu, lr);
@@ -214,8 +257,16 @@ cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote
   return cudaGetLastError();
 }
 
-cudaError_t launch_counter_apply(const int32_t* counter, float* x, uint64_t d, float lr, int8_t* opt_vote,
+cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, uint64_t d, float lr, int8_t* opt_vote,
                                  cudaStream_t st) {
+  if (packed) {
+    const uint32_t* cw = reinterpret_cast<const uint32_t*>(counter);
+    const bool vecp = aligned(x, 16) && (opt_vote == nullptr || aligned(opt_vote, 4));
+    if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, kSMs * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, kSMs * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    count_launch();
+    return cudaGetLastError();
+  }
   bool vec = aligned(x, 16) && aligned(counter, 16) && (opt_vote == nullptr || aligned(opt_vote, 4)) && d >= 4;
   if (vec) {
     counter_apply_kernel<true><<<grid_for(d / 4, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
@@ -244,9 +295,10 @@ cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint
   return cudaGetLastError();
 }
 
-cudaError_t launch_counter_apply_momentum(const int32_t* counter, float* x, float* v, uint64_t d, float mu, float lr,
-                                          int8_t* opt_vote, cudaStream_t st) {
-  counter_apply_momentum_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+cudaError_t launch_counter_apply_momentum(const int32_t* counter, bool packed, float* x, float* v, uint64_t d, float mu,
+                                          float lr, int8_t* opt_vote, cudaStream_t st) {
+  if (packed) counter_apply_momentum_kernel<true><<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+  else counter_apply_momentum_kernel<false><<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
   count_launch();
   return cudaGetLastError();
 }

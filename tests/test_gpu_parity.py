@@ -455,6 +455,23 @@ def test_step_replayed_from_a_cuda_graph(d, M, K):
     assert np.array_equal(bits(x.cpu().numpy()), bits(x_ref))
 
 
+@pytest.mark.parametrize("M,d,K", [(127, 40_003, 400), (128, 40_003, 400), (200, 20_001, 20_001), (130, 300_007, 9_000)])
+def test_many_workers_plain_and_byte_counters(M, d, K):
+    """Up to 127 workers the fused step counts votes in bytes, above that in int32: both sides of the switch,
+    with every worker voting the same way on some coordinates so that the counts reach +-M."""
+    s = W.spec("resnet18", d=d, M=M)
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    g[:, 5] = 1e3; g[:, 6] = -1e3; g[:, d - 1] = -1e3          # unanimous votes: counts +M, -M, -M
+    check_all(g, x, K, s.lr, tag=f"M={M}")
+    Kr = min(K, 1000)
+    ws = S.alloc_workspace(M, d, Kr, DEV)
+    xr = x.clone()
+    S.s3gd_step_randk(xr, g, Kr, s.lr, 3, 1, ws)
+    S.s3gd_device_status(ws)
+    x_o, _, _, _ = O.randk_step(x.cpu().numpy(), g.cpu().numpy(), Kr, s.lr, 3, 1)
+    assert np.array_equal(bits(xr.cpu().numpy()), bits(x_o))
+
+
 def test_majority_vote_semantics_and_range_flag():
     d, M, K = 10, 2, 4
     idx = torch.tensor([[1, 1, 3, 9], [1, 3, 4, 12]], dtype=torch.int32, device=DEV)
