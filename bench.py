@@ -60,7 +60,8 @@ def byte_models(M, d, K):
     words = (K + 31) // 32
     b_grad = 4 * M * d
     b_sel = 2 * M * (4 * K + 4 * words)
-    b_dense = b_grad + b_sel + 8 * d + 8 * d
+    b_count = 2 * d if M <= 127 else 8 * d        # vote counters cleared + read: bytes up to 127 workers, else int32
+    b_dense = b_grad + b_sel + b_count + 8 * d
     b_min = b_grad + 8 * min(d, M * K)
     return b_grad, b_dense, b_min
 

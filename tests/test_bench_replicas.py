@@ -45,7 +45,8 @@ def test_byte_models():
     import bench
     g, dense, mn = bench.byte_models(100, 11_173_962, 11_174)
     assert g == 4 * 100 * 11_173_962
-    assert dense == g + 2 * 100 * (4 * 11_174 + 4 * 350) + 16 * 11_173_962
+    assert dense == g + 2 * 100 * (4 * 11_174 + 4 * 350) + 10 * 11_173_962      # byte counters: 2d + x: 8d
+    assert bench.byte_models(128, 1000, 10)[1] == 4 * 128 * 1000 + 2 * 128 * (40 + 4) + 16 * 1000
     assert mn == g + 8 * 100 * 11_174
 
 
