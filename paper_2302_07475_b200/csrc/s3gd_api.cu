@@ -57,6 +57,9 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   L->off_seg = off;      off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
   L->off_segscan = off;  off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
   L->off_cand = off;     off = align_up(off + (size_t)M * L->cap * sizeof(uint2), 256);
+  // bin list of the two-pass selection: at most what one CTA's shared memory takes
+  L->bin_cap = L->cap < kSmallSelectBytes / 8u ? L->cap : kSmallSelectBytes / 8u;
+  L->off_bin = off;      off = align_up(off + (size_t)M * L->bin_cap * sizeof(uint2), 256);
   L->off_counter = off;  off = align_up(off + (size_t)d * sizeof(int32_t), 256);
   L->total = off;
   return true;

@@ -52,8 +52,9 @@ struct RowState {
   uint32_t exact;      // 1: this row uses the exact multi-pass route over the whole row
   uint32_t ticket_hist;   // blocks of the current histogram pass that have finished this row
   uint32_t ticket_count;  // blocks of the count pass that have finished this row
-  uint32_t done;          // 1: the single-CTA selection has already finished this row
-  uint32_t pad[5];
+  uint32_t done;          // 0: open; 1: finished by an on-chip selection; 2, 3: taken by the two-pass form (s3gd_select.cu)
+  uint32_t n_bin;         // entries collected so far in the row's bin list (two-pass form, votes only)
+  uint32_t pad[4];
 };
 
 // Byte offsets of the workspace regions; computed identically for sizing and use.
@@ -66,7 +67,8 @@ struct Layout {
   uint32_t n_sample;     // sampled entries per row
   uint32_t j_rank;       // sample rank that fixes tau_lo
   uint32_t sample_stride;  // distance between sampled groups of 8 (0: whole row sampled)
-  size_t off_hdr, off_rows, off_hist, off_seg, off_segscan, off_cand, off_counter, total;
+  uint32_t bin_cap;      // entries per row of the bin list (0: none)
+  size_t off_hdr, off_rows, off_hist, off_seg, off_segscan, off_cand, off_bin, off_counter, total;
 };
 
 bool make_layout(int M, uint64_t d, uint64_t K, Layout* L);
@@ -99,6 +101,11 @@ __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
+
+// RowState::done beyond 0 (open) and 1 (finished on chip): rows the two-pass form of the general
+// selection has taken (s3gd_select.cu).  kRowTwoPass: last histogram pass, count and emission follow;
+// kRowBin (votes only): the entries of the K-th magnitude's bin are collected and one CTA finishes them.
+constexpr uint32_t kRowTwoPass = 2u, kRowBin = 3u;
 
 // Does this row take its top-K from the filtered candidates (true) or from the whole row?
 __device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
@@ -165,6 +172,9 @@ struct EmitOut {
 };
 cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* cand, const uint2* seg, uint32_t* hdr,
                                 const EmitOut& o, cudaStream_t st);
+// Votes only, two-pass form: one CTA per row finishes the rows marked kRowBin from their bin lists
+cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t* hdr, const EmitOut& o,
+                              cudaStream_t st);
 // Votes only, rows too large for one SM: a cluster of 2 or 4 CTAs per row (cluster_size_for; 0 = none fits)
 uint32_t cluster_size_for(uint32_t n_cand);
 cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* cand, uint32_t* hdr, const EmitOut& o,

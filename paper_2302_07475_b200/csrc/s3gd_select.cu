@@ -73,23 +73,54 @@ __device__ __forceinline__ bool last_block_of_row(uint32_t* ticket, uint32_t n_b
 }
 
 // ------------------------------------------------------- histogram passes
-// Shared-memory histogram with warp-aggregated increments: lanes that hit the same
-// bin elect a leader which adds their count once (gradient magnitudes cluster in a
-// few bins, and quantised gradients do so in every pass, so plain atomics would
-// serialise on those bins).
+// Shared-memory histogram.  Gradient magnitudes cluster: in a coarse pass, or in any pass over
+// quantised gradients, a whole warp often holds one digit value, and 32 atomics on one word
+// would serialise.  So a warp first checks whether its active lanes agree (a ballot, a shuffle
+// and a vote); if so one lane adds their count.  Otherwise every lane adds for itself: the
+// digits are then spread out, and plain atomics measured faster than grouping equal digits
+// with __match_any_sync (two histogram passes over 10.8 M candidates: 77 against 87 us).
 __device__ __forceinline__ void hist_add(uint32_t* s_hist, bool on, uint32_t digit) {
-  const uint32_t peers = __match_any_sync(0xFFFFFFFFu, on ? digit : 0xFFFFFFFFu);
-  if (on && (peers & lanemask_lt()) == 0u) atomicAdd(&s_hist[digit], (uint32_t)__popc(peers));
+  const uint32_t act = __ballot_sync(0xFFFFFFFFu, on);
+  if (act == 0u) return;                             // warp-uniform
+  const uint32_t lead = (uint32_t)__ffs((int)act) - 1u;
+  const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, lead);
+  if (__all_sync(0xFFFFFFFFu, !on || digit == d0)) {
+    if ((threadIdx.x & 31u) == lead) atomicAdd(&s_hist[d0], (uint32_t)__popc(act));
+  } else if (on) {
+    atomicAdd(&s_hist[digit], 1u);
+  }
 }
 
 __device__ __forceinline__ bool in_prefix(uint32_t key, uint32_t prefix, int pass) {
   return pass == 0 || (key >> pass_shift(pass - 1)) == prefix;
 }
 
+// Two-pass form for rows that select from their candidates.  Every candidate is at or above
+// tau_lo, and the K-th magnitude is normally within a few percent of it, so the first two
+// digits of the three-pass form carry almost no information: all candidates share them.  The
+// first pass here takes the 11-bit digit from (key >> 10) - (tau_lo >> 10) instead -- 2047 bins
+// of 1024 keys, a quarter of an octave above tau_lo, and one bin for everything beyond -- and
+// thereby fixes the upper 21 bits at once; the second pass is the ordinary last pass over the
+// low 10 bits.  RowState::done == kRowTwoPass marks a row whose first pass found its bin; its
+// remaining passes run in launches that look only at such rows, and the general launch after
+// them skips it like any finished row.
+// If only the votes are wanted the rest is shorter still: everything above the bin is in the top K
+// whatever the low bits say, so it votes in the second sweep, which also copies the entries of the
+// bin itself -- a few thousand as a rule -- to the row's bin list; one CTA then selects the k_rem
+// largest of those on chip (ties to the lower index) and lets them vote.  No count, no ordered
+// emission.  The first pass knows how many entries the bin holds and marks the row kRowBin only
+// if the list fits one CTA's shared memory.
+constexpr uint32_t kJointClamp = (uint32_t)kHistBins - 1u;
+__device__ __forceinline__ uint32_t joint_digit(uint32_t key, uint32_t tau_lo) {
+  const uint32_t rel = (key >> pass_shift(1)) - (tau_lo >> pass_shift(1));
+  return rel < kJointClamp ? rel : kJointClamp;
+}
+
 // Find the digit in which the k_rem-th largest entry lies, fix it, and clear the
 // histogram for the next pass.  One block of kSelThreads threads.
 __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t row, uint32_t* __restrict__ h,
-                                           uint32_t* __restrict__ hdr, int pass, uint32_t* s_sum, uint32_t* s_sel) {
+                                           uint32_t* __restrict__ hdr, int pass, uint32_t* s_sum, uint32_t* s_sel,
+                                           bool joint = false, uint32_t bin_limit = 0u) {
   const uint32_t tid = threadIdx.x;
   const int nbins = 1 << pass_bits(pass);
   const int per = nbins / kSelThreads;               // 8 or 4 bins per thread, ascending
@@ -109,13 +140,24 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
   if (above < k_rem && above + mine >= k_rem) {      // exactly one thread
     uint32_t a = above;
     for (int i = per - 1; i >= 0; --i) {
-      if (a + c[i] >= k_rem) { s_sel[0] = tid * per + i; s_sel[1] = a; break; }
+      if (a + c[i] >= k_rem) { s_sel[0] = tid * per + i; s_sel[1] = a; s_sel[2] = c[i]; break; }
       a += c[i];
     }
   }
   __syncthreads();
   for (int i = 0; i < per; ++i) h[tid * per + i] = 0u;
-  if (tid == 0) {
+  if (tid == 0 && joint) {
+    // first pass of the two-pass form: the digit counts 1024-key steps above tau_lo.  The top bin
+    // collects everything further up; if the k_rem-th entry lies there the row stays untouched
+    // (prefix 0, k_rem K, histogram cleared) and the launch that follows the fast passes does it.
+    const uint32_t digit = s_sel[0], a = s_sel[1];
+    if (digit < kJointClamp) {
+      rows[row].prefix = (rows[row].tau_lo >> pass_shift(1)) + digit;
+      rows[row].k_rem = k_rem - a;
+      rows[row].done = s_sel[2] <= bin_limit ? kRowBin : kRowTwoPass;
+      atomicAdd(hdr + kHdrRowsDone, 1u);
+    }
+  } else if (tid == 0) {
     uint32_t digit = s_sel[0], a = s_sel[1];
     if (digit == 0xFFFFFFFFu) {                      // fewer than k_rem entries: cannot happen for a valid row
       atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
@@ -141,7 +183,7 @@ __device__ __forceinline__ void hist_pick_block(const uint32_t* __restrict__ gbi
                                                 uint32_t row, uint32_t gx) {
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_sum[kSelThreads];
-  __shared__ uint32_t s_sel[2];
+  __shared__ uint32_t s_sel[3];
   __shared__ uint32_t s_flag;
   const RowState rs = load_row_state<kFromL2>(rows + row);
   if (rs.done) return;                               // finished by the single-CTA selection (all blocks of the row agree)
@@ -205,6 +247,109 @@ __device__ __forceinline__ void hist_pick_block(const uint32_t* __restrict__ gbi
   }
   if (last_block_of_row(&rows[row].ticket_hist, gx, &s_flag))
     pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel);
+}
+
+// One block of a histogram pass of the two-pass form (pass 0: the joint digit; pass 2: the low
+// 10 bits).  Candidate rows only; a row has gx blocks.
+// The second sweep of a kRowBin row: entries above the bin vote, entries of the bin go to the list
+// (in any order).  A block stages its bin entries in shared memory and claims room in the list for
+// many of them at once: thousands of warps each adding to the one list counter of their row would
+// queue up on it (measured: 125 us for this sweep at 8,000 bin entries per row).
+constexpr int kTwoPassLoads = 4;                    // candidate entries a thread of a two-pass sweep has in flight
+constexpr uint32_t kBinStage = 512 + kTwoPassLoads * kSelThreads;   // staged entries; flushed before a round could overflow
+__device__ __forceinline__ void collect_bin_block(const uint2* __restrict__ c, const RowState& rs, RowState* rowp,
+                                                  uint2* __restrict__ bin, uint32_t bin_cap, const EmitOut& o,
+                                                  uint32_t bx, uint32_t gx) {
+  __shared__ uint2 s_stage[kBinStage];
+  __shared__ uint32_t s_n, s_base;
+  const uint32_t lane = threadIdx.x & 31, lt = lanemask_lt();
+  const uint32_t n = rs.n_cand, step = gx * kSelThreads * kTwoPassLoads;
+  if (threadIdx.x == 0) s_n = 0u;
+  __syncthreads();
+  for (uint32_t base = bx * kSelThreads * kTwoPassLoads; base < n; base += step) {      // block-uniform trip count
+    uint2 e[kTwoPassLoads];
+    bool on[kTwoPassLoads];
+#pragma unroll
+    for (int u = 0; u < kTwoPassLoads; ++u) {
+      const uint32_t i = base + u * kSelThreads + threadIdx.x;
+      on[u] = i < n;
+      e[u] = on[u] ? c[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < kTwoPassLoads; ++u) {
+      const uint32_t p = (e[u].x & kAbsMask) >> pass_shift(1);
+      if (on[u] && p > rs.prefix) add_vote(o.counter, o.packed, e[u].y, e[u].x >> 31);
+      const bool in_bin = on[u] && p == rs.prefix;
+      const uint32_t b = __ballot_sync(0xFFFFFFFFu, in_bin);
+      if (b == 0u) continue;                           // warp-uniform
+      const int lead = __ffs((int)b) - 1;
+      uint32_t at = 0;
+      if ((int)lane == lead) at = atomicAdd(&s_n, (uint32_t)__popc(b));
+      at = __shfl_sync(0xFFFFFFFFu, at, lead) + __popc(b & lt);
+      if (in_bin) s_stage[at] = e[u];
+    }
+    __syncthreads();
+    const uint32_t staged = s_n;
+    if (staged > kBinStage - (uint32_t)(kTwoPassLoads * kSelThreads) || (base + step >= n && staged != 0u)) {   // block-uniform
+      if (threadIdx.x == 0) s_base = atomicAdd(&rowp->n_bin, staged);
+      __syncthreads();
+      const uint32_t at0 = s_base;
+      for (uint32_t i = threadIdx.x; i < staged; i += kSelThreads)
+        if (at0 + i < bin_cap) bin[at0 + i] = s_stage[i];
+      __syncthreads();
+      if (threadIdx.x == 0) s_n = 0u;
+      __syncthreads();
+    }
+  }
+}
+
+__device__ __forceinline__ void hist_two_pass_block(const uint2* __restrict__ cand, uint32_t cap,
+                                                    RowState* __restrict__ rows, uint32_t K,
+                                                    uint32_t* __restrict__ hist, uint32_t* __restrict__ hdr, int pass,
+                                                    uint32_t bx, uint32_t row, uint32_t gx, uint2* __restrict__ bin,
+                                                    uint32_t bin_cap, const EmitOut& o) {
+  __shared__ uint32_t s_hist[kHistBins];
+  __shared__ uint32_t s_sum[kSelThreads];
+  __shared__ uint32_t s_sel[3];
+  __shared__ uint32_t s_flag;
+  const RowState rs = rows[row];
+  const bool joint = pass == 0;
+  if (!joint && rs.done == kRowBin) {
+    collect_bin_block(cand + (uint64_t)row * cap, rs, rows + row, bin + (uint64_t)row * bin_cap, bin_cap, o, bx, gx);
+    return;
+  }
+  if (joint ? (rs.done != 0u || !row_uses_candidates(rs, K, cap)) : rs.done != kRowTwoPass) return;
+  const int nbins = 1 << pass_bits(pass);
+  const uint32_t mask = (uint32_t)(nbins - 1);
+  uint32_t* g_hist = hist + (uint64_t)row * kHistBins;
+  if ((uint64_t)bx * kSelThreads * kTwoPassLoads < rs.n_cand) {
+    for (int b = threadIdx.x; b < nbins; b += kSelThreads) s_hist[b] = 0u;
+    __syncthreads();
+    const uint2* c = cand + (uint64_t)row * cap;
+    const uint32_t n = rs.n_cand, step = gx * kSelThreads * kTwoPassLoads;
+    for (uint32_t base = bx * kSelThreads * kTwoPassLoads; base < n; base += step) {
+      uint32_t key[kTwoPassLoads];
+      bool on[kTwoPassLoads];
+#pragma unroll
+      for (int u = 0; u < kTwoPassLoads; ++u) {
+        const uint32_t i = base + u * kSelThreads + threadIdx.x;
+        on[u] = i < n;
+        key[u] = on[u] ? (c[i].x & kAbsMask) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < kTwoPassLoads; ++u) {
+        if (joint) hist_add(s_hist, on[u], joint_digit(key[u], rs.tau_lo));
+        else hist_add(s_hist, on[u] && in_prefix(key[u], rs.prefix, pass), key[u] & mask);
+      }
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < nbins; b += kSelThreads) {
+      const uint32_t cnt = s_hist[b];
+      if (cnt) atomicAdd(&g_hist[b], cnt);
+    }
+  }
+  if (last_block_of_row(&rows[row].ticket_hist, gx, &s_flag))
+    pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel, joint, o.counter != nullptr && o.idx == nullptr ? bin_cap : 0u);
 }
 
 }  // namespace

@@ -160,11 +160,12 @@ __device__ __forceinline__ void count_scan_block(const uint32_t* __restrict__ gb
                                                  const uint2* __restrict__ cand, uint32_t cap,
                                                  const uint2* __restrict__ seg, RowState* __restrict__ rows,
                                                  uint32_t K, uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
-                                                 uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx) {
+                                                 uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx,
+                                                 uint32_t want_done = 0u) {
   __shared__ uint32_t s_gt[kWarpsPerTile], s_eq[kWarpsPerTile], s_warp[kSelThreads / 32];
   __shared__ uint32_t s_flag;
   const RowState rs = load_row_state<kFromL2>(rows + row);
-  if (rs.done) return;
+  if (rs.done != want_done) return;                  // 0: rows still open; kRowTwoPass: rows of the two-pass form
   const bool use_c = row_uses_candidates(rs, K, cap);
   const bool is_c = bx < gx_c;
   if (is_c && use_c) count_cand(cand, cap, seg, n_tiles, rs, row, bx, gx_c, cnt);
@@ -328,10 +329,11 @@ template <bool kFromL2>
 __device__ __forceinline__ void emit_block(const uint32_t* __restrict__ gbits, uint64_t d, uint32_t n_tiles,
                                            const uint2* __restrict__ cand, uint32_t cap, const uint2* __restrict__ seg,
                                            const uint2* __restrict__ scan, const RowState* __restrict__ rows,
-                                           const EmitOut& o, uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx) {
+                                           const EmitOut& o, uint32_t gx_c, uint32_t bx, uint32_t row, uint32_t gx,
+                                           uint32_t want_done = 0u) {
   __shared__ uint32_t s_wtot[kWarpsPerTile + 1];
   const RowState rs = load_row_state<kFromL2>(rows + row);
-  if (rs.done) return;
+  if (rs.done != want_done) return;
   const bool use_c = row_uses_candidates(rs, o.K, cap);
   const bool is_c = bx < gx_c;
   if (is_c && use_c) emit_cand(cand, cap, seg, scan, n_tiles, rs, row, bx, gx_c, o);
@@ -353,8 +355,18 @@ __global__ void __launch_bounds__(kSelThreads, 6) count_scan_kernel(const uint32
                                                                     uint32_t cap, const uint2* __restrict__ seg,
                                                                     RowState* __restrict__ rows, uint32_t K,
                                                                     uint2* __restrict__ cnt, uint32_t* __restrict__ hdr,
-                                                                    uint32_t gx_c) {
-  count_scan_block<false>(gbits, d, n_tiles, cand, cap, seg, rows, K, cnt, hdr, gx_c, blockIdx.x, blockIdx.y, gridDim.x);
+                                                                    uint32_t gx_c, uint32_t want_done) {
+  count_scan_block<false>(gbits, d, n_tiles, cand, cap, seg, rows, K, cnt, hdr, gx_c, blockIdx.x, blockIdx.y, gridDim.x,
+                          want_done);
+}
+
+__global__ void __launch_bounds__(kSelThreads, 6) hist_two_pass_kernel(const uint2* __restrict__ cand, uint32_t cap,
+                                                                       RowState* __restrict__ rows, uint32_t K,
+                                                                       uint32_t* __restrict__ hist,
+                                                                       uint32_t* __restrict__ hdr, int pass,
+                                                                       uint2* __restrict__ bin, uint32_t bin_cap,
+                                                                       EmitOut o) {
+  hist_two_pass_block(cand, cap, rows, K, hist, hdr, pass, blockIdx.x, blockIdx.y, gridDim.x, bin, bin_cap, o);
 }
 
 __global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
@@ -362,8 +374,9 @@ __global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __
                                                               uint32_t cap, const uint2* __restrict__ seg,
                                                               const uint2* __restrict__ scan,
                                                               const RowState* __restrict__ rows, EmitOut o,
-                                                              uint32_t gx_c) {
-  emit_block<false>(gbits, d, n_tiles, cand, cap, seg, scan, rows, o, gx_c, blockIdx.x, blockIdx.y, gridDim.x);
+                                                              uint32_t gx_c, uint32_t want_done) {
+  emit_block<false>(gbits, d, n_tiles, cand, cap, seg, scan, rows, o, gx_c, blockIdx.x, blockIdx.y, gridDim.x,
+                    want_done);
 }
 
 // The same passes as ONE cooperative launch -- three histogram passes, the counting pass and the
@@ -470,7 +483,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     if (!fits_single_cta(expect)) cluster = cluster_size_for(expect);
     if (cluster == 0u && !fits_single_cta(L.typical_cand)) cluster = cluster_size_for(L.typical_cand);
   }
-  if (use_filter) {
+  if (use_filter && (cluster != 0u || fits_single_cta(K))) {    // a candidate row has at least K candidates
     cudaError_t e = cluster ? launch_select_cluster(L, rows, cand, hdr, o, cluster, st)
                             : launch_select_small(L, rows, cand, seg, hdr, o, st);
     if (e != cudaSuccess) return e;
@@ -482,11 +495,40 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);
   const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * (only_fallback ? 4 : 8) + M - 1) / M);
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
+  // the sweeps of the two-pass form: all rows' blocks resident at once (six per SM), each with a longer
+  // run of candidates -- their per-block costs (row state, barriers, the ticket) weigh more than tail
+  // effects (resnet50 shape at K = 1 %: 64 blocks per row 0.826 ms, 27 per row 0.812 ms)
+  const uint32_t gx_two = clampu(((uint64_t)L.cap + 4095) / 4096, 1, clampu((uint64_t)kSMs * 6 / M, 8, 64));
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
   // With error compensation rows do run past the estimate (measured: the single launch then took
   // 1.07 ms where the five launches take 0.17 ms), so that mode keeps the five launches.
-  if (only_fallback && err_to_clear == nullptr) {
+  // Where the general passes carry the selection of candidate rows, those rows take the two-pass form
+  // first (two histogram launches instead of three, candidate blocks only); the single launch after it
+  // does whatever is left -- rows on the whole-row route, rows whose K-th magnitude lies more than a
+  // quarter octave above tau_lo -- and otherwise returns at once.
+  const bool two_pass = use_filter && !only_fallback && err_to_clear == nullptr;
+  if (two_pass) {
+    // bin lists only where the votes alone are wanted (the message needs positions)
+    uint2* bin = reinterpret_cast<uint2*>(base + L.off_bin);
+    const uint32_t bin_cap = votes_only ? L.bin_cap : 0u;
+    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 0, bin, bin_cap, o);
+    S3GD_CHECK_LAUNCH();
+    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 2, bin, bin_cap, o);
+    S3GD_CHECK_LAUNCH();
+    prof_mark(kPhaseThreshold, st);
+    if (bin_cap) {
+      cudaError_t e = launch_select_bin(L, rows, bin, hdr, o, st);
+      if (e != cudaSuccess) return e;
+    }
+    count_scan_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows, K, cnt,
+                                                                  hdr, gx_tile_c, kRowTwoPass);
+    S3GD_CHECK_LAUNCH();
+    emit_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
+                                                            gx_tile_c, kRowTwoPass);
+    S3GD_CHECK_LAUNCH();
+  }
+  if ((only_fallback || two_pass) && err_to_clear == nullptr) {
     // as many blocks as can be resident together, and no more than the largest pass has virtual blocks
     static int blocks_per_sm = 0;
     if (blocks_per_sm == 0) {
@@ -509,7 +551,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
                                                  dim3(kSelThreads), kargs, 0, st);
     if (ce != cudaSuccess) return ce;
     count_launch();
-    prof_mark(kPhaseThreshold, st);
+    if (!two_pass) prof_mark(kPhaseThreshold, st);
   } else {
     for (int pass = 0; pass < kNumPasses; ++pass) {
       hist_pick_kernel<<<dim3(gx_hist_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, rows, K,
@@ -518,10 +560,10 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     }
     prof_mark(kPhaseThreshold, st);
     count_scan_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows,
-                                                                         K, cnt, hdr, gx_tile_c);
+                                                                         K, cnt, hdr, gx_tile_c, 0u);
     S3GD_CHECK_LAUNCH();
     emit_kernel<<<dim3(gx_tile_c + gx_r, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
-                                                                   gx_tile_c);
+                                                                   gx_tile_c, 0u);
     S3GD_CHECK_LAUNCH();
   }
 #undef S3GD_CHECK_LAUNCH

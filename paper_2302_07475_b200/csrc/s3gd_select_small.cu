@@ -49,18 +49,23 @@ __device__ __forceinline__ uint32_t block_scan_excl_1024(uint32_t v, uint32_t* s
 // kMaxTiesUnordered of them, beyond that by a radix select on the index.
 constexpr uint32_t kMaxTiesUnordered = 1024;
 
-template <bool kOrdered>
+// kBin (votes only): the list is the row's bin list of the two-pass form (s3gd_select.cu) instead of
+// its candidates -- the entries that share the upper 21 bits of the K-th magnitude -- of which the
+// k_rem largest are kept; everything above them has voted already and the row is counted as finished.
+template <bool kOrdered, bool kBin = false>
 __global__ void __launch_bounds__(kSmallThreads, 1)
 select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand, uint32_t cap,
                     const uint2* __restrict__ seg, uint32_t n_tiles, uint32_t* __restrict__ hdr, EmitOut o) {
+  static_assert(!(kOrdered && kBin), "bin lists are unordered");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_warp[kSmallWarps];
   __shared__ uint32_t s_sel[2];
   const uint32_t row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, lt = lanemask_lt();
   const RowState rs = rows[row];
-  if (!row_uses_candidates(rs, o.K, cap) || !fits_single_cta(rs.n_cand)) return;
-  const uint32_t n = rs.n_cand;
+  if (kBin ? rs.done != kRowBin : (!row_uses_candidates(rs, o.K, cap) || !fits_single_cta(rs.n_cand))) return;
+  const uint32_t n = kBin ? (rs.n_bin < cap ? rs.n_bin : cap) : rs.n_cand;
+  const uint32_t k_want = kBin ? rs.k_rem : o.K;     // entries to keep out of the n
   uint32_t* s_bits = reinterpret_cast<uint32_t*>(smem_raw);   // [n] bit patterns, in ascending index order
   uint32_t* s_idx = s_bits + n;                               // [n] their indices
   const uint2* c = cand + (uint64_t)row * cap;
@@ -122,7 +127,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   }
 
   // ---- radix select: tau = K-th largest magnitude, take = how many entries equal to tau are kept
-  uint32_t prefix = 0, k_rem = o.K, n_equal = 0;
+  uint32_t prefix = 0, k_rem = k_want, n_equal = 0;
   for (int pass = 0; pass < kNumPasses; ++pass) {
     const int nbins = 1 << pass_bits(pass);
     const uint32_t mask = (uint32_t)(nbins - 1);
@@ -265,7 +270,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
         s_tie_neg[slot] = bits >> 31;
       }
     }
-    uint32_t n_kept = o.K;
+    uint32_t n_kept = k_want;
     if (rank_ties) {
       __syncthreads();
       const uint32_t e = s_sel[0];                               // == n_equal
@@ -283,14 +288,16 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     if (tid == 0) {
       rows[row].tau = tau;
       rows[row].take_ties = take;
-      rows[row].n_emitted = n_kept;
-      rows[row].done = 1u;
-      atomicAdd(hdr + kHdrRowsDone, 1u);
-      if (n_kept != o.K) {
+      rows[row].n_emitted = kBin ? (n_kept == k_want ? o.K : n_kept) : n_kept;
+      if (!kBin) {                                               // a kRowBin row was counted when it was marked
+        rows[row].done = 1u;
+        atomicAdd(hdr + kHdrRowsDone, 1u);
+      }
+      if (n_kept != k_want || (kBin && rs.n_bin > cap)) {
         atomicAdd(hdr + kHdrBadCount, 1u);
         atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
       }
-      atomicMax(hdr + kHdrMaxCand, n);
+      atomicMax(hdr + kHdrMaxCand, kBin ? rs.n_cand : n);
     }
     return;
   }
@@ -541,6 +548,17 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
   if (e != cudaSuccess) return e;
   kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, cand, L.cap, seg, L.n_tiles, hdr, o);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) count_launch();
+  return e;
+}
+
+cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t* hdr, const EmitOut& o,
+                              cudaStream_t st) {
+  auto kernel = select_small_kernel<false, true>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
+  if (e != cudaSuccess) return e;
+  kernel<<<L.M, kSmallThreads, (size_t)L.bin_cap * 8u, st>>>(rows, bin, L.bin_cap, nullptr, 0u, hdr, o);
   e = cudaGetLastError();
   if (e == cudaSuccess) count_launch();
   return e;

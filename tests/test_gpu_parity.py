@@ -296,6 +296,37 @@ def test_ties_at_the_threshold_in_a_row_that_needs_a_cluster(n_ties, take):
     assert info[1] == 0 and info[4] > 27_136     # served from the candidates, more of them than one SM holds
 
 
+@pytest.mark.parametrize("shape", ["gap", "octave_edge", "smooth"])
+@pytest.mark.parametrize("d,K", [(4_000_000, 40_000), (12_000_000, 120_000)])
+def test_rows_selected_by_the_general_passes(shape, d, K):
+    """Rows with more survivors than the on-chip selections hold (the larger size also for the votes-only step).
+
+    Their first histogram pass counts 1024-key steps above the filter threshold, a quarter octave in all.
+    "gap": the K-th magnitude lies two orders of magnitude above the threshold, outside that range, so
+    the rows are finished by the launch that follows; "octave_edge": magnitudes around 2.0, where the
+    exponent changes between the threshold and the K-th magnitude; "smooth": a Gaussian tail.
+    """
+    M = 3
+    g = torch.Generator("cpu").manual_seed(d // 1000 + K + len(shape))
+    rows = []
+    for m in range(M):
+        if shape == "gap":
+            v = 0.5 + 0.5 * torch.rand(d, generator=g)
+            perm = torch.randperm(d, generator=g)
+            n_big = K + K // 10
+            v[perm[:n_big]] = 100.0 + 100.0 * torch.rand(n_big, generator=g)
+        elif shape == "octave_edge":
+            v = 2.02327 * torch.rand(d, generator=g)              # the top 1.15 % lies above 2.0, the K-th is 1 %
+        else:
+            v = torch.randn(d, generator=g).abs()
+        sign = torch.where(torch.rand(d, generator=g) < 0.5, -1.0, 1.0)
+        rows.append((v * sign).float())
+    grads = torch.stack(rows).contiguous().to(DEV)
+    x = torch.zeros(d, device=DEV)
+    info = check_all(grads, x, K, 0.25, tag=f"general passes {shape} d={d}")
+    assert info[1] == 0 and info[4] > 27_136     # served from the candidates, more of them than one SM holds
+
+
 # ------------------------------------------- error compensation and momentum (s3gd_step_ex)
 @pytest.mark.parametrize("K,eta,mu", [(300, 1.0, None), (300, 0.5, 0.9), (75_002, 1.0, None), (300_007, 1.0, 0.5),
                                       (0, 1.0, 0.5), (3_000, 0.0, None)])
