@@ -127,8 +127,9 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   }
 
   // ---- radix select: tau = K-th largest magnitude, take = how many entries equal to tau are kept
-  uint32_t prefix = 0, k_rem = k_want, n_equal = 0;
-  for (int pass = 0; pass < kNumPasses; ++pass) {
+  // (the entries of a bin list share their upper 21 bits, which the first sweep fixed: last pass only)
+  uint32_t prefix = kBin ? rs.prefix : 0u, k_rem = k_want, n_equal = 0;
+  for (int pass = kBin ? kNumPasses - 1 : 0; pass < kNumPasses; ++pass) {
     const int nbins = 1 << pass_bits(pass);
     const uint32_t mask = (uint32_t)(nbins - 1);
     for (int b = tid; b < nbins; b += kSmallThreads) s_hist[b] = 0u;

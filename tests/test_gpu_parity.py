@@ -199,6 +199,12 @@ def test_large_full_size_row_by_row():
     vote_o, _ = O.majority_vote(idx_o, sgn_o, s.M, K, s.d)
     x_o = O.apply_vote(x0, vote_o, s.lr)
     assert np.array_equal(bits(x.cpu().numpy()), bits(x_o))
+    del idx, sgn
+    x2 = torch.from_numpy(x0).to(DEV)              # the votes-only step takes another route through the selection
+    S.s3gd_step(x2, g, K, s.lr, ws)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0
+    assert np.array_equal(bits(x2.cpu().numpy()), bits(x_o))
 
 
 def test_large_recipe_reduced_64bit_offsets():
@@ -296,7 +302,7 @@ def test_ties_at_the_threshold_in_a_row_that_needs_a_cluster(n_ties, take):
     assert info[1] == 0 and info[4] > 27_136     # served from the candidates, more of them than one SM holds
 
 
-@pytest.mark.parametrize("shape", ["gap", "octave_edge", "smooth"])
+@pytest.mark.parametrize("shape", ["gap", "octave_edge", "smooth", "tie_group"])
 @pytest.mark.parametrize("d,K", [(4_000_000, 40_000), (12_000_000, 120_000)])
 def test_rows_selected_by_the_general_passes(shape, d, K):
     """Rows with more survivors than the on-chip selections hold (the larger size also for the votes-only step).
@@ -304,7 +310,9 @@ def test_rows_selected_by_the_general_passes(shape, d, K):
     Their first histogram pass counts 1024-key steps above the filter threshold, a quarter octave in all.
     "gap": the K-th magnitude lies two orders of magnitude above the threshold, outside that range, so
     the rows are finished by the launch that follows; "octave_edge": magnitudes around 2.0, where the
-    exponent changes between the threshold and the K-th magnitude; "smooth": a Gaussian tail.
+    exponent changes between the threshold and the K-th magnitude; "smooth": a Gaussian tail;
+    "tie_group": more entries exactly at the K-th magnitude than one CTA's shared memory holds, a third
+    of them kept, so the votes-only step too must count and emit in index order.
     """
     M = 3
     g = torch.Generator("cpu").manual_seed(d // 1000 + K + len(shape))
@@ -315,6 +323,13 @@ def test_rows_selected_by_the_general_passes(shape, d, K):
             perm = torch.randperm(d, generator=g)
             n_big = K + K // 10
             v[perm[:n_big]] = 100.0 + 100.0 * torch.rand(n_big, generator=g)
+        elif shape == "tie_group":
+            v = 0.9 * torch.rand(d, generator=g)
+            perm = torch.randperm(d, generator=g)
+            n_ties = (5 * K) // 6
+            n_big = K - n_ties // 3
+            v[perm[:n_big]] = 5.0 + torch.rand(n_big, generator=g)
+            v[perm[n_big:n_big + n_ties]] = 2.0
         elif shape == "octave_edge":
             v = 2.02327 * torch.rand(d, generator=g)              # the top 1.15 % lies above 2.0, the K-th is 1 %
         else:
