@@ -252,21 +252,20 @@ __device__ __forceinline__ void hist_pick_block(const uint32_t* __restrict__ gbi
 // One block of a histogram pass of the two-pass form (pass 0: the joint digit; pass 2: the low
 // 10 bits).  Candidate rows only; a row has gx blocks.
 // The second sweep of a kRowBin row: entries above the bin vote, entries of the bin go to the list
-// (in any order).  A block stages its bin entries in shared memory and claims room in the list for
-// many of them at once: thousands of warps each adding to the one list counter of their row would
-// queue up on it (measured: 125 us for this sweep at 8,000 bin entries per row).
+// (in any order).  Each warp stages its bin entries in shared memory and claims room in the list
+// for 64 or more of them at once: one claim per warp and step queued 8,000 atomics per row on the
+// one list counter (125 us for this sweep), and staging per block cost a barrier per round (61 us).
 constexpr int kTwoPassLoads = 4;                    // candidate entries a thread of a two-pass sweep has in flight
-constexpr uint32_t kBinStage = 512 + kTwoPassLoads * kSelThreads;   // staged entries; flushed before a round could overflow
+constexpr uint32_t kBinFlush = 64;                   // a warp flushes once it holds more than this
+constexpr uint32_t kBinStage = kBinFlush + kTwoPassLoads * 32;   // ... so that a round of loads always fits
 __device__ __forceinline__ void collect_bin_block(const uint2* __restrict__ c, const RowState& rs, RowState* rowp,
                                                   uint2* __restrict__ bin, uint32_t bin_cap, const EmitOut& o,
                                                   uint32_t bx, uint32_t gx) {
-  __shared__ uint2 s_stage[kBinStage];
-  __shared__ uint32_t s_n, s_base;
-  const uint32_t lane = threadIdx.x & 31, lt = lanemask_lt();
+  __shared__ uint2 s_stage[kSelThreads / 32][kBinStage];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, lt = lanemask_lt();
   const uint32_t n = rs.n_cand, step = gx * kSelThreads * kTwoPassLoads;
-  if (threadIdx.x == 0) s_n = 0u;
-  __syncthreads();
-  for (uint32_t base = bx * kSelThreads * kTwoPassLoads; base < n; base += step) {      // block-uniform trip count
+  uint32_t staged = 0;                               // warp-uniform
+  for (uint32_t base = bx * kSelThreads * kTwoPassLoads; base < n; base += step) {
     uint2 e[kTwoPassLoads];
     bool on[kTwoPassLoads];
 #pragma unroll
@@ -282,23 +281,18 @@ __device__ __forceinline__ void collect_bin_block(const uint2* __restrict__ c, c
       const bool in_bin = on[u] && p == rs.prefix;
       const uint32_t b = __ballot_sync(0xFFFFFFFFu, in_bin);
       if (b == 0u) continue;                           // warp-uniform
-      const int lead = __ffs((int)b) - 1;
-      uint32_t at = 0;
-      if ((int)lane == lead) at = atomicAdd(&s_n, (uint32_t)__popc(b));
-      at = __shfl_sync(0xFFFFFFFFu, at, lead) + __popc(b & lt);
-      if (in_bin) s_stage[at] = e[u];
+      if (in_bin) s_stage[warp][staged + __popc(b & lt)] = e[u];
+      staged += (uint32_t)__popc(b);
     }
-    __syncthreads();
-    const uint32_t staged = s_n;
-    if (staged > kBinStage - (uint32_t)(kTwoPassLoads * kSelThreads) || (base + step >= n && staged != 0u)) {   // block-uniform
-      if (threadIdx.x == 0) s_base = atomicAdd(&rowp->n_bin, staged);
-      __syncthreads();
-      const uint32_t at0 = s_base;
-      for (uint32_t i = threadIdx.x; i < staged; i += kSelThreads)
-        if (at0 + i < bin_cap) bin[at0 + i] = s_stage[i];
-      __syncthreads();
-      if (threadIdx.x == 0) s_n = 0u;
-      __syncthreads();
+    if (staged > kBinFlush || (staged != 0u && base + step >= n)) {     // warp-uniform
+      __syncwarp();
+      uint32_t at0 = 0;
+      if (lane == 0) at0 = atomicAdd(&rowp->n_bin, staged);
+      at0 = __shfl_sync(0xFFFFFFFFu, at0, 0);
+      for (uint32_t i = lane; i < staged; i += 32)
+        if (at0 + i < bin_cap) bin[at0 + i] = s_stage[warp][i];
+      __syncwarp();
+      staged = 0;
     }
   }
 }
