@@ -319,6 +319,13 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_kernel(const
 // is cheaper than a vote and four ballots per iteration; survivors are staged per CTA.
 constexpr int kStageCap = 512;                 // survivors staged per tile (8 bytes each, two buffers)
 
+// (row, tile) of a persistent CTA's next work item, gridDim.x items further on
+__device__ __forceinline__ void next_tile(uint32_t& row, uint32_t& t, uint32_t n_tiles) {
+  uint64_t nt = (uint64_t)t + gridDim.x;
+  while (nt >= n_tiles) { nt -= n_tiles; ++row; }
+  t = (uint32_t)nt;
+}
+
 template <bool kEF>
 __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(const uint32_t* __restrict__ gbits, int M, uint64_t d,
                                                               RowState* __restrict__ rows, uint2* __restrict__ cand,
@@ -333,8 +340,10 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
   uint32_t pend_n = 0, pend_row = 0, pend_t = 0;   // staged survivors of the previous tile (uniform)
   uint32_t pend_base = 0;                          // thread 0: the claim made for them (may still be in flight)
   int par = 0;
-  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x, par ^= 1) {
-    const uint32_t row = (uint32_t)(w / n_tiles), t = (uint32_t)(w - (uint64_t)row * n_tiles);
+  // walk (row, tile) without dividing in the loop (a 64-bit division per tile is a few percent of
+  // the instructions of this issue-bound kernel)
+  uint32_t row = (uint32_t)(blockIdx.x / n_tiles), t = (uint32_t)(blockIdx.x - (uint64_t)row * n_tiles);
+  for (uint64_t w = blockIdx.x; w < n_work; w += gridDim.x, par ^= 1, next_tile(row, t, n_tiles)) {
     const uint32_t* rowp = gbits + (uint64_t)row * d;
     const uint32_t head = row_head(rowp, d);
     const float tau = __uint_as_float(rows[row].tau_lo);
