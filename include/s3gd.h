@@ -17,7 +17,8 @@
  *    "host" means ordinary host memory.  The library never allocates, frees or
  *    retains a pointer.  Every buffer, including the workspace, is the caller's.
  *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
- *    the default stream).  No call synchronises except s3gd_device_status().
+ *    the default stream).  No call synchronises except s3gd_device_status(),
+ *    s3gd_last_device_status() and s3gd_profile_end().
  *  - Magnitude order is the unsigned order of the fp32 bit pattern with the sign
  *    bit cleared.  Denormals are not flushed; NaN and Inf order by bit pattern.
  *  - Exactly K entries are kept per worker; equal magnitudes go to the lower
@@ -25,9 +26,18 @@
  *  - Indices are 0-based uint32 and ascending within a worker.  Sign bit j of a
  *    worker belongs to its j-th index: word j/32, bit j%32 (LSB first),
  *    1 = negative; unused bits of the last word are 0.
- *  - Return value: S3GD_OK or an error detected on the host BEFORE anything is
- *    enqueued (outputs untouched).  Conditions only the device can see are
- *    recorded in the workspace and read back with s3gd_device_status().
+ *  - Return value: S3GD_OK, or an argument / workspace error detected on the host
+ *    BEFORE anything is enqueued (outputs untouched).  S3GD_ERR_CUDA reports a failed
+ *    CUDA runtime call and may come after part of the call's work was enqueued: the
+ *    outputs are then undefined.  Conditions only the device can see are recorded
+ *    in the workspace and read back with s3gd_device_status().
+ *  - Limits: 1 <= M <= 65535 workers, 1 <= d < 2^32 coordinates, 0 <= K <= d.
+ *  - Threads: calls on different workspaces may be made from different host threads
+ *    (the only shared host state is a set of per-device caches that are written once).
+ *    Calls that share a workspace must be ordered by the caller.  Not thread-safe:
+ *    the s3gd_profile_* calls (one session per process; do not open or close one while
+ *    another thread is inside a step) and s3gd_majority_vote_noalloc (one built-in
+ *    scratch array per device).
  */
 #ifndef S3GD_H_
 #define S3GD_H_
@@ -47,9 +57,10 @@ extern "C" {
 
 typedef enum s3gd_status {
   S3GD_OK = 0,
-  S3GD_ERR_INVALID_ARG = 1, /* NULL pointer, M <= 0, d == 0, d >= 2^32, K > d, bad alignment */
+  S3GD_ERR_INVALID_ARG = 1, /* NULL pointer, M <= 0, M > 65535, d == 0, d >= 2^32, K > d, bad alignment */
   S3GD_ERR_WORKSPACE = 2,   /* workspace NULL, smaller than s3gd_workspace_bytes(), or not 256-byte aligned */
-  S3GD_ERR_CUDA = 3,        /* a CUDA runtime call failed (launch error, wrong device, ...) */
+  S3GD_ERR_CUDA = 3,        /* a CUDA runtime call failed (launch error, wrong device, no room to load the
+                               library's GPU code, ...); outputs may be partly written */
   S3GD_ERR_INDEX_RANGE = 4, /* device: an index >= d was given to s3gd_majority_vote (skipped) */
   S3GD_ERR_INTERNAL = 5,    /* device: a selection did not produce exactly K entries */
   S3GD_ERR_TOO_LARGE = 6    /* s3gd_majority_vote_noalloc: d exceeds s3gd_noalloc_max_d() */
@@ -188,6 +199,30 @@ S3GD_API s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64
  *   [4] largest candidate count of a row  [5..7] reserved (0)
  */
 S3GD_API s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* info);
+/* The same without the counters: s3gd_device_status(ws, stream, NULL). */
+S3GD_API s3gd_status s3gd_last_device_status(const void* ws, void* stream);
+
+/*
+ * Test hooks for the exactness safety net (the paper has no counterpart).
+ *
+ * For 0 < K <= d/4 the selection reads each gradient row once: a threshold taken at a fixed
+ * rank of a 65,536-entry sample of the row filters the row, and the top K are then found
+ * among the survivors.  A row whose filter kept fewer than K entries (threshold too high) or
+ * more than the workspace has room for (too low) is redone exactly over the whole row; that
+ * decision is taken per row on the device, and with a sound sampling rank it is almost never
+ * needed.  These two calls are s3gd_topk_sign and s3gd_step with the sampling rank given by
+ * the caller, so that a test can force either failure on ordinary data: sample_rank = 1 puts
+ * the threshold at the largest sampled magnitude (too few survivors), a rank near 65,536 puts
+ * it at the smallest (too many).  sample_rank = 0 means the library's own rank.  The results
+ * must be, and are checked to be, identical to those of the ordinary calls; info[1] of
+ * s3gd_device_status counts the rows that were redone.  Workspace as for the ordinary calls.
+ */
+S3GD_API s3gd_status s3gd_debug_topk_sign(const float* grads, int M, uint64_t d, uint64_t K,
+                                          uint32_t* out_idx, uint32_t* out_signbits,
+                                          void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank);
+S3GD_API s3gd_status s3gd_debug_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr,
+                                     uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
+                                     void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank);
 
 /*
  * Majority vote without any caller-provided scratch (the paper has no counterpart: this is
@@ -197,19 +232,27 @@ S3GD_API s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* 
  * another framework's callback that must not call into its allocator, a plug-in that is
  * handed nothing but input and output buffers, a process whose device memory is already
  * fully owned by a pool it does not control.  The d int32 counters live in a fixed array
- * inside this library (16 MiB + 256 bytes on every GPU that loads it, held until the
- * process exits), so d is limited: s3gd_noalloc_max_d() = 4,194,304 coordinates; a larger
- * d returns S3GD_ERR_TOO_LARGE and nothing is enqueued.  The call allocates and frees
- * nothing.
+ * inside this library's GPU code (16 MiB + 256 bytes per GPU), so d is limited:
+ * s3gd_noalloc_max_d() = 4,194,304 coordinates; a larger d returns S3GD_ERR_TOO_LARGE and
+ * nothing is enqueued.  The call itself calls no allocation routine and frees nothing.
+ *
+ * When the array's memory is taken: not when the library is loaded into the process.  The
+ * CUDA runtime loads GPU code lazily by default, so the 16 MiB (and the code of the two
+ * kernels the call uses) are reserved on a device by the FIRST call made there, and are then
+ * held until the process exits.  Make that first call -- any small vote will do -- while the
+ * device still has that much free memory; if it does not, the first call returns
+ * S3GD_ERR_CUDA and can be repeated later.  Running the process with
+ * CUDA_MODULE_LOADING=EAGER moves the reservation to the creation of the CUDA context.
  *
  *  idx, signbits, M, K, d, out_vote   as for s3gd_majority_vote (dev pointers)
  *  opt_bad_count  dev or NULL  receives the number of indices >= d that were skipped
  *
- * The first call on each device looks up the device address of the built-in array (a
- * runtime query, no allocation) with that device current; make that first call outside
- * any stream capture.  All calls on a device share the one array: it is cleared at the
- * start of every call, so results never depend on earlier calls, but two calls that may
- * run on the GPU at the same time (different streams) race on it -- serialise them.
+ * The first call on each device also looks up the device address of the built-in array (a
+ * runtime query) with that device current; make that first call outside any stream
+ * capture.  All calls on a device share the one array: it is cleared at the start of every
+ * call, so results never depend on earlier calls, but two calls that may run on the GPU at
+ * the same time (different streams) race on it -- serialise them.  Not thread-safe: do not
+ * make the first call on a device from two host threads at once.
  */
 S3GD_API uint64_t s3gd_noalloc_max_d(void);
 S3GD_API s3gd_status s3gd_majority_vote_noalloc(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K,

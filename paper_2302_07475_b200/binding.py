@@ -25,7 +25,8 @@ STATUS_NAMES = {
 EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd_majority_vote",
            "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
            "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
-           "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter")
+           "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter", "s3gd_last_device_status",
+           "s3gd_debug_topk_sign", "s3gd_debug_step")
 
 
 class S3gdError(RuntimeError):
@@ -83,6 +84,12 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_randk_sign.argtypes = [vp, ctypes.c_int, u64, u64, u32, u32, u32p, u32p, vp, sz, vp]
     lib.s3gd_step_randk.restype = ctypes.c_int
     lib.s3gd_step_randk.argtypes = [vp, vp, ctypes.c_int, u64, u64, ctypes.c_float, u32, u32, u32p, u32p, vp, vp, sz, vp]
+    lib.s3gd_last_device_status.restype = ctypes.c_int
+    lib.s3gd_last_device_status.argtypes = [vp, vp]
+    lib.s3gd_debug_topk_sign.restype = ctypes.c_int
+    lib.s3gd_debug_topk_sign.argtypes = lib.s3gd_topk_sign.argtypes + [u32]
+    lib.s3gd_debug_step.restype = ctypes.c_int
+    lib.s3gd_debug_step.argtypes = lib.s3gd_step.argtypes + [u32]
     if path is None:
         _lib = lib
     return lib
@@ -182,6 +189,40 @@ def s3gd_device_status(ws: torch.Tensor, raise_on_error: bool = True):
     if raise_on_error:
         _check("s3gd_device_status", code)
     return code, list(info)
+
+
+def s3gd_last_device_status(ws: torch.Tensor) -> int:
+    """Synchronises the current stream; returns the status code recorded by the kernels (0 = ok)."""
+    w = _ptr(ws, torch.uint8, name="ws")
+    with torch.cuda.device(ws.device):
+        return int(load().s3gd_last_device_status(w, _stream(ws)))
+
+
+def s3gd_debug_topk_sign(grads: torch.Tensor, K: int, out_idx: torch.Tensor, out_signbits: torch.Tensor,
+                         ws: torch.Tensor, sample_rank: int) -> None:
+    """s3gd_topk_sign with the sampling rank of the filter threshold forced (0: the library's own)."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (g, M, d, K, _ptr(out_idx, torch.int32, M * K, "out_idx"),
+            _ptr(out_signbits, torch.int32, M * words(K), "out_signbits"),
+            _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(grads.device):
+        code = load().s3gd_debug_topk_sign(*args, _stream(grads), int(sample_rank))
+    _check("s3gd_debug_topk_sign", code)
+
+
+def s3gd_debug_step(x: torch.Tensor, grads: torch.Tensor, K: int, lr: float, ws: torch.Tensor, sample_rank: int,
+                    opt_idx: Optional[torch.Tensor] = None, opt_signbits: Optional[torch.Tensor] = None,
+                    opt_vote: Optional[torch.Tensor] = None) -> None:
+    """s3gd_step with the sampling rank of the filter threshold forced (0: the library's own)."""
+    g = _ptr(grads, torch.float32, name="grads")
+    M, d = grads.shape
+    args = (_ptr(x, torch.float32, d, "x"), g, M, d, K, ctypes.c_float(lr),
+            _ptr(opt_idx, torch.int32, M * K, "opt_idx"), _ptr(opt_signbits, torch.int32, M * words(K), "opt_signbits"),
+            _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(x.device):
+        code = load().s3gd_debug_step(*args, _stream(x), int(sample_rank))
+    _check("s3gd_debug_step", code)
 
 
 PHASES = ("sample", "filter", "threshold", "emit", "apply")

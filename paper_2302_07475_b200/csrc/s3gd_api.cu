@@ -2,6 +2,8 @@
 // the kernels of each call are enqueued.  See include/s3gd.h for the contract.
 #include <math.h>
 
+#include <atomic>
+
 #include "s3gd_common.cuh"
 
 namespace s3gd {
@@ -65,6 +67,35 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   return true;
 }
 
+// ------------------------------------------------------- per-device host caches
+// Filled on first use and never changed afterwards; two threads that race on the first use
+// store the same value, so relaxed atomics are enough.
+namespace {
+std::atomic<int> g_sm_count[kMaxDevices];
+}  // namespace
+
+int sm_count() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return kDefaultSMs;
+  int n = g_sm_count[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = kDefaultSMs;
+    g_sm_count[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
+cudaError_t opt_in_dynamic_smem(const void* func, int bytes, int* done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < kMaxDevices;
+  if (cached && __atomic_load_n(&done[dev], __ATOMIC_RELAXED) >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && cached) __atomic_store_n(&done[dev], bytes, __ATOMIC_RELAXED);
+  return e;
+}
+
 // ---------------------------------------------------------------- profiling
 namespace {
 struct Profiler {
@@ -72,8 +103,8 @@ struct Profiler {
   bool filter_only = false;           // record only the two marks around the filter pass
   int max_steps = 0, n_steps = 0;
   cudaEvent_t* ev = nullptr;          // kPhaseMarks events per recorded step
-  unsigned long long launches = 0;
 } g_prof;
+std::atomic<unsigned long long> g_launches{0};   // kernels enqueued while a profiling session is open
 }  // namespace
 
 void prof_mark(int phase, cudaStream_t st) {
@@ -83,7 +114,9 @@ void prof_mark(int phase, cudaStream_t st) {
   if (phase == kPhaseApplied) ++g_prof.n_steps;
 }
 
-void count_launch(int n) { g_prof.launches += (unsigned long long)n; }
+void count_launch(int n) {
+  if (g_prof.on) g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed);
+}
 
 namespace {
 
@@ -127,10 +160,19 @@ size_t s3gd_workspace_bytes(int M, uint64_t d, uint64_t K) {
   return make_layout(M, d, K, &L) ? L.total : 0;
 }
 
-s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
-                           uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream) {
+namespace {
+// sample_rank != 0 replaces the sampling plan's rank (the debug entry points); the workspace
+// layout, and with it the candidate capacity, stays that of the plan.
+void override_sample_rank(Layout* L, uint32_t sample_rank) {
+  if (sample_rank == 0u || L->cap == 0u) return;
+  L->j_rank = sample_rank < L->n_sample ? sample_rank : L->n_sample;
+}
+
+s3gd_status topk_sign_impl(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
+                           uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank) {
   Layout L;
   if (!make_layout(M, d, K, &L) || grads == nullptr || !aligned(grads, 4)) return S3GD_ERR_INVALID_ARG;
+  override_sample_rank(&L, sample_rank);
   if (K > 0 && (out_idx == nullptr || out_signbits == nullptr || !aligned(out_idx, 4) || !aligned(out_signbits, 4)))
     return S3GD_ERR_INVALID_ARG;
   s3gd_status s = check_ws(L, ws, ws_bytes);
@@ -144,6 +186,18 @@ s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, ui
   }
   S3GD_TRY(cudaMemsetAsync(out_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
   return from_cuda(launch_select(grads, L, ws, out_idx, out_signbits, nullptr, false, nullptr, nullptr, 0.f, st));
+}
+}  // namespace
+
+s3gd_status s3gd_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
+                           uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream) {
+  return topk_sign_impl(grads, M, d, K, out_idx, out_signbits, ws, ws_bytes, stream, 0u);
+}
+
+s3gd_status s3gd_debug_topk_sign(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
+                                 uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream,
+                                 uint32_t sample_rank) {
+  return topk_sign_impl(grads, M, d, K, out_idx, out_signbits, ws, ws_bytes, stream, sample_rank);
 }
 
 s3gd_status s3gd_majority_vote(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
@@ -227,16 +281,31 @@ s3gd_status check_step_args(const float* x, const float* grads, uint32_t* opt_id
 
 }  // namespace
 
-s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
-                      uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
+namespace {
+s3gd_status plain_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
+                       uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream,
+                       uint32_t sample_rank) {
   Layout L;
   if (!make_layout(M, d, K, &L)) return S3GD_ERR_INVALID_ARG;
+  override_sample_rank(&L, sample_rank);
   s3gd_status s = check_step_args(x, grads, opt_idx, opt_signbits);
   if (s != S3GD_OK) return s;
   s = check_ws(L, ws, ws_bytes);
   if (s != S3GD_OK) return s;
   return step_impl(x, grads, nullptr, nullptr, 0.f, M, d, K, lr, opt_idx, opt_signbits, opt_vote, L, ws,
                    static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
+                      uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
+  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, 0u);
+}
+
+s3gd_status s3gd_debug_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
+                            uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream,
+                            uint32_t sample_rank) {
+  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, sample_rank);
 }
 
 s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta, float* opt_v, float mu, int M,
@@ -335,7 +404,7 @@ s3gd_status profile_begin(int max_steps, bool filter_only) {
   }
   g_prof.max_steps = max_steps;
   g_prof.n_steps = 0;
-  g_prof.launches = 0;
+  g_launches.store(0);
   g_prof.filter_only = filter_only;
   g_prof.on = true;
   return S3GD_OK;
@@ -360,7 +429,7 @@ s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches) {
     }
   }
   if (n_steps) *n_steps = g_prof.n_steps;
-  if (launches) *launches = g_prof.launches;
+  if (launches) *launches = g_launches.load();
   for (size_t i = 0; i < (size_t)g_prof.max_steps * kPhaseMarks; ++i) cudaEventDestroy(g_prof.ev[i]);
   delete[] g_prof.ev;
   g_prof = Profiler();
@@ -379,5 +448,7 @@ s3gd_status s3gd_device_status(const void* ws, void* stream, uint32_t* info) {
   if (h[kHdrStatus] & kFlagIndexRange) return S3GD_ERR_INDEX_RANGE;
   return S3GD_OK;
 }
+
+s3gd_status s3gd_last_device_status(const void* ws, void* stream) { return s3gd_device_status(ws, stream, nullptr); }
 
 }  // extern "C"

@@ -25,7 +25,14 @@ __host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
 constexpr int kSampleBins = 32768;                 // magnitude >> 16: sign-less bf16 pattern
 constexpr uint32_t kAbsMask = 0x7FFFFFFFu;
 
-constexpr int kSMs = 148;                          // B200
+constexpr int kDefaultSMs = 148;                   // B200; used only if the device query fails
+constexpr int kMaxDevices = 64;                    // per-device host caches are this long
+
+// SMs of the current device (asked once per device).  Grids are sized in multiples of it.
+int sm_count();
+// cudaFuncSetAttribute(func, MaxDynamicSharedMemorySize, bytes), issued once per device and
+// kernel: `done` is a zero-initialised array of kMaxDevices flags owned by the call site.
+cudaError_t opt_in_dynamic_smem(const void* func, int bytes, int* done);
 
 // --------------------------------------------------------------- device state
 // Header at the start of the workspace (64 x uint32).

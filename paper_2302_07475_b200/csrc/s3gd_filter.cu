@@ -442,14 +442,15 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
   auto sample = ef_err ? sample_threshold_kernel<true> : sample_threshold_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(sample, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static int opted[2][kMaxDevices];
+  cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(sample), (int)smem, opted[ef_err ? 1 : 0]);
   if (e != cudaSuccess) return e;
   // clearing blocks: the SMs the M sampling blocks leave idle, and never fewer than 32
   unsigned n_clear = 0;
   if (zero_counter) {
-    const unsigned used = (unsigned)L.M % (unsigned)kSMs;
-    n_clear = (unsigned)kSMs - used;
-    if (n_clear < 32u) n_clear += (unsigned)kSMs;
+    const unsigned used = (unsigned)L.M % (unsigned)sm_count();
+    n_clear = (unsigned)sm_count() - used;
+    if (n_clear < 32u) n_clear += (unsigned)sm_count();
   }
   sample<<<(unsigned)L.M + n_clear, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
                                                       (uint32_t)L.K, hdr, hist, ef_err, eta, (uint32_t)L.M, zero_counter,
@@ -459,7 +460,7 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   prof_mark(kPhaseSampled, st);
   count_launch(2);
   const uint64_t n_work = (uint64_t)L.M * L.n_tiles;
-  const uint64_t blocks = n_work < (uint64_t)kSMs * 8 ? n_work : (uint64_t)kSMs * 8;
+  const uint64_t blocks = n_work < (uint64_t)sm_count() * 8 ? n_work : (uint64_t)sm_count() * 8;
   const bool dense = (uint64_t)L.typical_cand * 250u > L.d;
   auto filter = dense ? (ef_err ? filter_scan_kernel<true> : filter_scan_kernel<false>)
                       : (ef_err ? filter_kernel<true> : filter_kernel<false>);

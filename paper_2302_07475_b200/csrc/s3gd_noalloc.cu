@@ -14,27 +14,34 @@ namespace {
 
 constexpr uint64_t kStaticMaxD = S3GD_NOALLOC_MAX_D;
 
-// 256 bytes of status words followed by the counters.  Lives for the life of the process
-// on every device that loads the library (16 MiB + 256 B).  Shared by all calls.
+// 256 bytes of status words followed by the counters (16 MiB + 256 B).  Shared by all calls.
+// The array is part of this file's GPU code module.  The CUDA runtime loads a module on a device
+// when something in it is first used there (lazy loading, the default since CUDA 12.2), and that is
+// when the device memory of the array is reserved; from then on it is held until the process exits.
 static __device__ __align__(256) uint32_t g_static_scratch[kHdrWords + kStaticMaxD];
 
-constexpr int kMaxDevices = 64;
-uint32_t* g_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device; set on first use
+// device address of g_static_scratch, per device; set on first use.  Threads that race on the
+// first use ask the same question and store the same answer.
+uint32_t* g_scratch_addr[kMaxDevices];
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address the GPU
 // can use; the device address has to be asked for, once per device, with that device current.
+// This query is also what makes the runtime load the module (see above): if the device has no
+// room left for the array and the kernels, it fails here and the caller reports S3GD_ERR_CUDA.
 cudaError_t scratch_address(uint32_t** out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (g_scratch_addr[dev] == nullptr) {
+  uint32_t* addr = __atomic_load_n(&g_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (addr == nullptr) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_scratch);
     if (e != cudaSuccess) return e;
-    g_scratch_addr[dev] = static_cast<uint32_t*>(p);
+    addr = static_cast<uint32_t*>(p);
+    __atomic_store_n(&g_scratch_addr[dev], addr, __ATOMIC_RELEASE);
   }
-  *out = g_scratch_addr[dev];
+  *out = addr;
   return cudaSuccess;
 }
 

@@ -89,7 +89,7 @@ cudaError_t launch_randk(const float* grads, int M, uint64_t d, uint64_t K, uint
   while ((1ull << (2 * h)) < d) ++h;
   const uint64_t warps = (uint64_t)M * ((K + 31) / 32);
   uint64_t blocks = (warps + 7) / 8;
-  const uint64_t cap = (uint64_t)kSMs * 8;
+  const uint64_t cap = (uint64_t)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   randk_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(grads), M, (uint32_t)d, (uint32_t)K,
                                                  h, seed, step, out_idx, out_signbits, counter, packed ? 1u : 0u, hdr);

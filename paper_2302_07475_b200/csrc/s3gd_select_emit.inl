@@ -463,7 +463,7 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
                            : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, packed, st);
     if (e != cudaSuccess) return e;
   } else {
-    init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, kSMs * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
+    init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, sm_count() * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
     S3GD_CHECK_LAUNCH();
     prof_mark(kPhaseSampled, st);
   }
@@ -493,12 +493,12 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   // odd row that did not fit or fell back to the whole-row route, and normally exit at once:
   // keep them small.  Otherwise they carry the selection of all rows: about eight CTAs per SM.
   const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);
-  const uint32_t per_row = (uint32_t)(((uint64_t)kSMs * (only_fallback ? 4 : 8) + M - 1) / M);
+  const uint32_t per_row = (uint32_t)(((uint64_t)sm_count() * (only_fallback ? 4 : 8) + M - 1) / M);
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   // the sweeps of the two-pass form: all rows' blocks resident at once (six per SM), each with a longer
   // run of candidates -- their per-block costs (row state, barriers, the ticket) weigh more than tail
   // effects (resnet50 shape at K = 1 %: 64 blocks per row 0.826 ms, 27 per row 0.812 ms)
-  const uint32_t gx_two = clampu(((uint64_t)L.cap + 4095) / 4096, 1, clampu((uint64_t)kSMs * 6 / M, 8, 64));
+  const uint32_t gx_two = clampu(((uint64_t)L.cap + 4095) / 4096, 1, clampu((uint64_t)sm_count() * 6 / M, 8, 64));
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
   // With error compensation rows do run past the estimate (measured: the single launch then took
@@ -530,16 +530,19 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   }
   if ((only_fallback || two_pass) && err_to_clear == nullptr) {
     // as many blocks as can be resident together, and no more than the largest pass has virtual blocks
-    static int blocks_per_sm = 0;
+    // (the occupancy of a kernel is a property of the device: asked once per device, and two threads
+    //  that ask at the same time store the same number)
+    static int occupancy[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int blocks_per_sm = __atomic_load_n(&occupancy[dev], __ATOMIC_RELAXED);
     if (blocks_per_sm == 0) {
       cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, general_passes_kernel, kSelThreads, 0);
       if (e != cudaSuccess) return e;
       if (blocks_per_sm < 1) return cudaErrorLaunchOutOfResources;
+      __atomic_store_n(&occupancy[dev], blocks_per_sm, __ATOMIC_RELAXED);
     }
-    int n_sm = 0, dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return cudaErrorUnknown;
+    const int n_sm = sm_count();
     GeneralArgs ga;
     ga.gbits = gbits; ga.d = L.d; ga.n_tiles = L.n_tiles; ga.cand = cand; ga.cap = L.cap; ga.seg = seg; ga.cnt = cnt;
     ga.rows = rows; ga.K = K; ga.hist = hist; ga.hdr = hdr; ga.o = o; ga.M = (uint32_t)M;

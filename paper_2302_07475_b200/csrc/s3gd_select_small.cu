@@ -546,7 +546,8 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
   if (need > kSmallSelectBytes) need = kSmallSelectBytes;
   const bool ordered = o.idx != nullptr || o.signbits != nullptr || o.counter == nullptr;
   auto kernel = ordered ? select_small_kernel<true> : select_small_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
+  static int opted[2][kMaxDevices];
+  cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)kSmallSelectBytes, opted[ordered ? 1 : 0]);
   if (e != cudaSuccess) return e;
   kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, cand, L.cap, seg, L.n_tiles, hdr, o);
   e = cudaGetLastError();
@@ -557,7 +558,8 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
 cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t* hdr, const EmitOut& o,
                               cudaStream_t st) {
   auto kernel = select_small_kernel<false, true>;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
+  static int opted[kMaxDevices];
+  cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)kSmallSelectBytes, opted);
   if (e != cudaSuccess) return e;
   kernel<<<L.M, kSmallThreads, (size_t)L.bin_cap * 8u, st>>>(rows, bin, L.bin_cap, nullptr, 0u, hdr, o);
   e = cudaGetLastError();
@@ -581,7 +583,9 @@ cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* 
                                   uint32_t cluster, cudaStream_t st) {
   auto kernel = cluster == 2u ? select_cluster_kernel<2> : (cluster == 4u ? select_cluster_kernel<4> : select_cluster_kernel<8>);
   if (cluster != 2u && cluster != 4u && cluster != 8u) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallSelectBytes);
+  static int opted[3][kMaxDevices];
+  cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)kSmallSelectBytes,
+                                      opted[cluster == 2u ? 0 : (cluster == 4u ? 1 : 2)]);
   if (e != cudaSuccess) return e;
   uint64_t need = (uint64_t)((L.cap + cluster - 1) / cluster) * 8u;
   if (need > kSmallSelectBytes) need = kSmallSelectBytes;

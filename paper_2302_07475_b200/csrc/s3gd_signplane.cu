@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(256) signplane_counts_kernel(const float* __re
 
 inline unsigned blocks_for(uint64_t threads) {
   uint64_t b = (threads + 255) / 256;
-  uint64_t cap = (uint64_t)kSMs * 8;
+  uint64_t cap = (uint64_t)sm_count() * 8;
   if (b < 1) b = 1;
   return (unsigned)(b < cap ? b : cap);
 }

@@ -230,13 +230,13 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cudaStream_t st) {
   if (aligned(x, 16) && aligned(vote, 16) && d >= 16) {
     uint64_t n16 = d / 16;
-    apply_kernel_v16<<<grid_for(n16, 256, kSMs * 8), 256, 0, st>>>(x, vote, n16, lr);
+    apply_kernel_v16<<<grid_for(n16, 256, sm_count() * 8), 256, 0, st>>>(x, vote, n16, lr);
     count_launch();
     uint64_t done = n16 * 16;
     if (done < d) apply_kernel<<<1, 256, 0, st>>>(x + done, vote + done, d - done, lr);
     if (done < d) count_launch();
   } else {
-    apply_kernel<<<grid_for(d, 256, kSMs * 8), 256, 0, st>>>(x, vote, d, lr);
+    apply_kernel<<<grid_for(d, 256, sm_count() * 8), 256, 0, st>>>(x, vote, d, lr);
     count_launch();
   }
   return cudaGetLastError();
@@ -246,13 +246,13 @@ cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, i
                                 int32_t* counter, uint32_t* hdr, cudaStream_t st) {
   uint64_t total = (uint64_t)M * K;
   if (total == 0) return cudaSuccess;
-  vote_scatter_kernel<<<grid_for(total, 256, kSMs * 16), 256, 0, st>>>(idx, signbits, M, K, d, counter, hdr);
+  vote_scatter_kernel<<<grid_for(total, 256, sm_count() * 16), 256, 0, st>>>(idx, signbits, M, K, d, counter, hdr);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st) {
-  counter_sign_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, d, vote);
+  counter_sign_kernel<<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, d, vote);
   count_launch();
   return cudaGetLastError();
 }
@@ -262,17 +262,17 @@ cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, 
   if (packed) {
     const uint32_t* cw = reinterpret_cast<const uint32_t*>(counter);
     const bool vecp = aligned(x, 16) && (opt_vote == nullptr || aligned(opt_vote, 4));
-    if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, kSMs * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
-    else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, kSMs * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
     count_launch();
     return cudaGetLastError();
   }
   bool vec = aligned(x, 16) && aligned(counter, 16) && (opt_vote == nullptr || aligned(opt_vote, 4)) && d >= 4;
   if (vec) {
-    counter_apply_kernel<true><<<grid_for(d / 4, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
+    counter_apply_kernel<true><<<grid_for(d / 4, 256, sm_count() * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
     count_launch();
   } else {
-    counter_apply_kernel<false><<<grid_for(d, 256, kSMs * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
+    counter_apply_kernel<false><<<grid_for(d, 256, sm_count() * 8), 256, 0, st>>>(counter, x, d, lr, opt_vote);
     count_launch();
   }
   return cudaGetLastError();
@@ -281,7 +281,7 @@ cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, 
 cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint64_t n, cudaStream_t st) {
   if (aligned(err, 16) && aligned(grads, 16) && n >= 4) {
     const uint64_t n4 = n / 4;
-    ef_accumulate_kernel_v4<<<grid_for(n4, 256, kSMs * 16), 256, 0, st>>>(reinterpret_cast<float4*>(err),
+    ef_accumulate_kernel_v4<<<grid_for(n4, 256, sm_count() * 16), 256, 0, st>>>(reinterpret_cast<float4*>(err),
                                                                          reinterpret_cast<const float4*>(grads), eta, n4);
     count_launch();
     if (n4 * 4 < n) {
@@ -289,7 +289,7 @@ cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint
       count_launch();
     }
   } else {
-    ef_accumulate_kernel<<<grid_for(n, 256, kSMs * 16), 256, 0, st>>>(err, grads, eta, n);
+    ef_accumulate_kernel<<<grid_for(n, 256, sm_count() * 16), 256, 0, st>>>(err, grads, eta, n);
     count_launch();
   }
   return cudaGetLastError();
@@ -297,15 +297,15 @@ cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint
 
 cudaError_t launch_counter_apply_momentum(const int32_t* counter, bool packed, float* x, float* v, uint64_t d, float mu,
                                           float lr, int8_t* opt_vote, cudaStream_t st) {
-  if (packed) counter_apply_momentum_kernel<true><<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
-  else counter_apply_momentum_kernel<false><<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+  if (packed) counter_apply_momentum_kernel<true><<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+  else counter_apply_momentum_kernel<false><<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
                                   cudaStream_t st) {
-  apply_momentum_kernel<<<grid_for(d, 256, kSMs * 16), 256, 0, st>>>(x, v, vote, d, mu, lr);
+  apply_momentum_kernel<<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(x, v, vote, d, mu, lr);
   count_launch();
   return cudaGetLastError();
 }

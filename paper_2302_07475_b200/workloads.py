@@ -176,6 +176,17 @@ def make_grads(s: WorkloadSpec, device, step: int = 0,
     return out
 
 
+def make_rows(s: WorkloadSpec, rows, device, step: int = 0) -> torch.Tensor:
+    """[len(rows), d]: the listed workers' rows of make_grads(s, device, step), without drawing the others."""
+    device = torch.device(device)
+    rows = list(rows)
+    out = torch.empty((len(rows), s.d), dtype=torch.float32, device=device)
+    blocks = block_scales(s, device) if s.n_blocks else None
+    for i, m in enumerate(rows):
+        _fill_row(s, out[i], int(m), step, blocks)
+    return out
+
+
 def make_x(s: WorkloadSpec, device) -> torch.Tensor:
     """[d] fp32 parameters, N(0, x_sigma^2)."""
     device = torch.device(device)

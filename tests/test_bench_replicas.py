@@ -43,11 +43,34 @@ def test_single_rank_is_identity():
 
 def test_byte_models():
     import bench
-    g, dense, mn = bench.byte_models(100, 11_173_962, 11_174)
+    b = bench.byte_models(100, 11_173_962, 11_174)
+    g = b["grad"]
+    msg = 2 * 100 * (4 * 11_174 + 4 * 350)
     assert g == 4 * 100 * 11_173_962
-    assert dense == g + 2 * 100 * (4 * 11_174 + 4 * 350) + 10 * 11_173_962      # byte counters: 2d + x: 8d
-    assert bench.byte_models(128, 1000, 10)[1] == 4 * 128 * 1000 + 2 * 128 * (40 + 4) + 16 * 1000
-    assert mn == g + 8 * 100 * 11_174
+    assert b["dense"] == g + msg + 10 * 11_173_962      # byte counters: 2d + x: 8d
+    assert b["json"] == g + msg + 16 * 11_173_962       # int32 counters: 8d + x: 8d
+    assert b["moved"] == g + 10 * 11_173_962            # no message in the fused step
+    assert bench.byte_models(128, 1000, 10)["dense"] == 4 * 128 * 1000 + 2 * 128 * (40 + 4) + 16 * 1000
+    assert b["min"] == g + 8 * 100 * 11_174
+    # the published table's figures for the headline shape (GB, three decimals)
+    assert round(b["json"] / 1e9, 3) == 4.658 and round(b["min"] / 1e9, 3) == 4.479
+    f = bench.fractions(b, 1.0, 6457.4)
+    assert abs(f["json"]["GBps"] - b["json"] / 1e6) < 1e-6 and abs(f["json"]["of_8TBps"] - f["json"]["GBps"] / 8000) < 1e-12
+
+
+def test_repeats_cover_about_a_second():
+    import bench
+    assert bench.pick_repeats(7, 20, 0.76) == 7                 # asked for
+    assert bench.pick_repeats(0, 20, 0.76) == 50                # 20 x 0.76 ms regions: capped
+    assert bench.pick_repeats(0, 300, 0.76) == 5                # long regions: the floor
+    assert bench.pick_repeats(0, 5, 12.0) == 17
+
+
+def test_make_rows_matches_make_grads():
+    from paper_2302_07475_b200 import workloads as W
+    s = W.spec("resnet18", d=5_003, M=6)
+    full = W.make_grads(s, "cpu")
+    assert torch.equal(W.make_rows(s, [4, 1], "cpu"), full[[4, 1]])
 
 
 def test_reference_arm_other_ranks_do_nothing():

@@ -174,9 +174,32 @@ def test_resnet50_tie_stress_full_size():
     _full_size("resnet50_ties", W.SPECS["resnet50_ties"].Ks, sample_rows=(31,))
 
 
-@pytest.mark.skipif(os.environ.get("S3GD_TEST_LARGE") != "1", reason="67 GB case: set S3GD_TEST_LARGE=1")
+def _room_for_large_case():
+    """The d = 2.1e9, M = 8 case holds 67.2 GB of gradients, x twice, 8.7 GB of workspace and the message on
+    the device, and one 8.4 GB row plus the oracle's temporaries (about five times that) on the host."""
+    free_dev, _ = torch.cuda.mem_get_info()
+    need_dev = 100e9
+    if free_dev < need_dev:
+        return f"device has {free_dev / 1e9:.0f} GB free, the case needs {need_dev / 1e9:.0f} GB"
+    try:
+        import psutil
+        free_host = psutil.virtual_memory().available
+    except Exception:
+        return ""
+    need_host = 60e9
+    if free_host < need_host:
+        return f"host has {free_host / 1e9:.0f} GB available, the oracle needs {need_host / 1e9:.0f} GB for one row"
+    return ""
+
+
 def test_large_full_size_row_by_row():
     """d = 2.1e9, M = 8: the rows are generated, stepped and then certified one by one on the host."""
+    if os.environ.get("S3GD_TEST_LARGE") == "0":
+        pytest.skip("switched off with S3GD_TEST_LARGE=0")
+    why = _room_for_large_case()
+    if why:
+        print("large case skipped:", why)
+        pytest.skip(why)
     s = W.SPECS["large"]
     K = s.Ks[0]
     g = W.make_grads(s, DEV)
@@ -222,6 +245,20 @@ def test_large_recipe_reduced_64bit_offsets():
     i_o, s_o = O.topk_sign_threshold(g_last[None, :], K)
     assert np.array_equal(u32(idx)[s.M - 1], i_o[0]) and np.array_equal(u32(sgn)[s.M - 1], s_o[0])
     assert O.check_topk_sign_row(g_last, K, u32(idx)[s.M - 1], u32(sgn)[s.M - 1]) == ""
+    del g_last
+    # the votes-only fused step (the route the benchmark times for the large workload: bin lists, no
+    # message) over the same rows: every row's oracle selection, then the oracle's vote and update
+    idx_o = np.zeros((s.M, K), np.uint32); sgn_o = np.zeros((s.M, S.binding.words(K)), np.uint32)
+    for m in range(s.M):
+        i_o, s_o = O.topk_sign_threshold(g[m].cpu().numpy()[None, :], K)
+        idx_o[m], sgn_o[m] = i_o[0], s_o[0]
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o)
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, s.M, K, s.d)
+    x_o = O.apply_vote(x.cpu().numpy(), vote_o, s.lr)
+    S.s3gd_step(x, g, K, s.lr, ws)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0
+    assert np.array_equal(bits(x.cpu().numpy()), bits(x_o))
 
 
 # ------------------------------------------------------------------ edge cases
@@ -258,6 +295,53 @@ def test_rows_that_leave_the_single_read_route():
     g[1] = torch.randn(d, device=DEV)
     info = check_all(g, torch.zeros(d, device=DEV), K, 0.1, tag="mixed")
     assert info[1] == M - 1
+
+
+@pytest.mark.parametrize("name,d,M,K", [("resnet18", 300_007, 7, 3_001), ("resnet18", 11_173_962, 6, 11_174),
+                                        ("resnet50_ties", 25_557_032, 3, 255_570), ("large", 4_000_003, 3, 30_000)])
+@pytest.mark.parametrize("sample_rank,side", [(1, "too few"), (65_536, "too many")])
+def test_forced_bad_threshold_takes_the_whole_row_route(name, d, M, K, sample_rank, side):
+    """Rows longer than the sample (d > 131,072), ordinary data, and a sampling rank that is far off.
+
+    Rank 1 puts the filter threshold at the largest sampled magnitude, so fewer than K entries survive;
+    rank 65,536 puts it at the smallest, so more survive than the candidate list holds.  Either way every
+    row must notice on the device, redo its selection over the whole row, and give the oracle's answer:
+    this is what makes the single-read design exact whatever the sample says.  Checked for the message
+    alone, the fused step with outputs and the votes-only fused step (three different kernel sequences)."""
+    s = W.spec(name, d=d, M=M)
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    gn = g.cpu().numpy()
+    idx_o, sgn_o = O.topk_sign_threshold(gn, K)
+    i_d, s_d = O.topk_sign(gn[M - 1:M], K)                        # the definition itself on one row
+    assert np.array_equal(i_d[0], idx_o[M - 1]) and np.array_equal(s_d[0], sgn_o[M - 1])
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, M, K, d)
+    x_o = O.apply_vote(x.cpu().numpy(), vote_o, s.lr)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    ws.fill_(0x3C)
+    idx = torch.full((M, K), -1, dtype=torch.int32, device=DEV)
+    sgn = torch.full((M, S.binding.words(K)), -1, dtype=torch.int32, device=DEV)
+    vote = torch.full((d,), 77, dtype=torch.int8, device=DEV)
+    S.s3gd_debug_topk_sign(g, K, idx, sgn, ws, sample_rank)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == M, f"{side}: {info[1]} of {M} rows were redone"
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"{side}: message differs"
+    idx.fill_(-1); sgn.fill_(-1)
+    xa = x.clone()
+    S.s3gd_debug_step(xa, g, K, s.lr, ws, sample_rank, idx, sgn, vote)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == M
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o) and np.array_equal(vote.cpu().numpy(), vote_o)
+    assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"{side}: fused step with outputs differs"
+    xb = x.clone()
+    S.s3gd_debug_step(xb, g, K, s.lr, ws, sample_rank)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == M
+    assert np.array_equal(bits(xb.cpu().numpy()), bits(x_o)), f"{side}: votes-only fused step differs"
+    # rank 0 is the ordinary call: nothing is redone
+    xc = x.clone()
+    S.s3gd_debug_step(xc, g, K, s.lr, ws, 0)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0 and np.array_equal(bits(xc.cpu().numpy()), bits(x_o))
 
 
 @pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900), (5_000, 2_500), (1025, 1)])

@@ -7,7 +7,9 @@ process whose GPU memory already belongs to a pool it does not own.  Its counter
 fixed array inside the library, shared by every call, so the interesting failure is a
 second call that sees what the first one left behind.  The test therefore makes two calls
 in a row -- the second on a different, much sparser message -- and requires each result to
-equal s3gd_majority_vote's on the same inputs exactly (votes are integers: tolerance 0).
+equal s3gd_majority_vote's on the same inputs exactly (votes are integers: tolerance 0), and
+both to equal the CPU oracle's vote, so that a mistake the two library calls share (they use the
+same two kernels) cannot hide.
 """
 import ctypes
 
@@ -16,6 +18,7 @@ import pytest
 import torch
 
 import paper_2302_07475_b200 as S
+from oracle import s3gd_oracle as O
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -37,6 +40,8 @@ def _both(idx, sgn, M, K, d):
     bad = torch.full((1,), -1, dtype=torch.int32, device=DEV)
     S.s3gd_majority_vote_noalloc(idx, sgn, M, K, d, got, bad)
     torch.cuda.synchronize()
+    want, want_bad = O.majority_vote(idx.cpu().numpy().view(np.uint32), sgn.cpu().numpy().view(np.uint32), M, K, d)
+    assert np.array_equal(got.cpu().numpy(), want) and int(bad.item()) == want_bad, "differs from the oracle's vote"
     return ref.cpu().numpy(), got.cpu().numpy(), int(bad.item())
 
 
