@@ -26,8 +26,10 @@ Readings where the paper is silent (all listed in the design notes):
 * the update is one fp32 round-to-nearest operation: x - lr or x + lr.
 
 All integer results are exact, so GPU output must equal them bit for bit.
-Also here: error compensation (Eq. (5)-(6)), the momentum update (Section 4.7) and the
-random-K variant (Section 3.4, Algorithm 2).
+Also here: error compensation (Eq. (5)-(6)), the momentum update (Section 4.7), the
+random-K variant (Section 3.4, Algorithm 2), and the server's message to the workers
+(Section 2.2, "Majority vote": the voted ternary vector, zero outside the union of the
+workers' supports) in two transmitted forms with the paper's bit counts beside them.
 
 Parity status: every function below is pinned by tests that do not call it to
 build their expectation (brute-force rank counting, the printed worked
@@ -257,6 +259,85 @@ def randk_step(x: np.ndarray, grads: np.ndarray, K: int, lr, seed: int, step: in
     idx, sgn = randk_sign(grads, K, seed, step)
     vote, _ = majority_vote(idx, sgn, M, K, d)
     return apply_vote(x, vote, lr), idx, sgn, vote
+
+
+# --------------------------------------------------------------------------
+# The server's side of the exchange (Section 2.2, "Majority vote", and Algorithm 1's
+# "send"/"receive" lines): vote counts as sums, and the voted vector in the two forms
+# in which it can travel back to the workers.
+# --------------------------------------------------------------------------
+
+def vote_counts(idx: np.ndarray, signbits: np.ndarray, M: int, K: int, d: int) -> np.ndarray:
+    """count[n] = sum over workers of their vote on coordinate n (+1, -1 or nothing), as int64.
+
+    majority_vote() is the sign of this.  Sums of several groups of workers add up to the
+    sum of all of them, which is what lets a server be split over coordinate ranges."""
+    idx = np.asarray(idx, dtype=np.uint32).reshape(M, K)
+    signbits = np.asarray(signbits, dtype=np.uint32).reshape(M, (K + 31) // 32)
+    count = np.zeros(d, dtype=np.int64)
+    for m in range(M):
+        for j in range(K):
+            n = int(idx[m, j])
+            if n < d:
+                neg = (int(signbits[m, j >> 5]) >> (j & 31)) & 1
+                count[n] += -1 if neg else 1
+    return count
+
+
+def encode_vote_2bit(vote: np.ndarray) -> np.ndarray:
+    """Dense form: two bits per coordinate, 16 coordinates per uint32 word, LSB first.
+
+    Bit 0 of a pair says "moved", bit 1 says "negative": 0 -> 00, +1 -> 01, -1 -> 11.
+    Padding pairs of the last word are 00."""
+    v = np.asarray(vote, dtype=np.int8)
+    d = v.shape[0]
+    words = np.zeros((d + 15) // 16, dtype=np.uint32)
+    for n in range(d):
+        code = 0 if v[n] == 0 else (1 if v[n] > 0 else 3)
+        words[n >> 4] |= np.uint32(code << (2 * (n & 15)))
+    return words
+
+
+def decode_vote_2bit(words: np.ndarray, d: int) -> np.ndarray:
+    """Inverse of encode_vote_2bit (the pair 10 never occurs; it decodes as 0)."""
+    w = np.asarray(words, dtype=np.uint32)
+    vote = np.zeros(d, dtype=np.int8)
+    for n in range(d):
+        code = (int(w[n >> 4]) >> (2 * (n & 15))) & 3
+        vote[n] = 1 if code == 1 else (-1 if code == 3 else 0)
+    return vote
+
+
+def encode_vote_sparse(vote: np.ndarray):
+    """Sparse form: the non-zero coordinates, ascending, and their sign bits -- the same
+    layout as a worker's message (uint32 indices; bit j of the sign words belongs to
+    index j, LSB first, 1 = negative, zero padding).  Returns (idx [n], signbits [ceil(n/32)])."""
+    v = np.asarray(vote, dtype=np.int8)
+    where = [n for n in range(v.shape[0]) if v[n] != 0]
+    idx = np.array(where, dtype=np.uint32)
+    return idx, pack_sign_bits(np.array([v[n] < 0 for n in where], dtype=bool))
+
+
+def decode_vote_sparse(idx: np.ndarray, signbits: np.ndarray, d: int) -> np.ndarray:
+    """Inverse of encode_vote_sparse.  An index >= d is ignored."""
+    vote = np.zeros(d, dtype=np.int8)
+    idx = np.asarray(idx, dtype=np.uint32)
+    sb = np.asarray(signbits, dtype=np.uint32)
+    for j in range(idx.shape[0]):
+        n = int(idx[j])
+        if n < d:
+            vote[n] = -1 if (int(sb[j >> 5]) >> (j & 31)) & 1 else 1
+    return vote
+
+
+def uplink_bits(K: int, N: int) -> float:
+    """Bits one worker sends per round as Section 2.2 counts them: K + K log2(N / K)."""
+    return 0.0 if K == 0 else K + K * float(np.log2(N / K))
+
+
+def downlink_bits(n_voted: int, N: int) -> float:
+    """Bits the server sends per round as Section 2.2 counts them: |N^t| + |N^t| log2(N / |N^t|)."""
+    return uplink_bits(n_voted, N)
 
 
 # --------------------------------------------------------------------------

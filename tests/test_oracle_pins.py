@@ -248,6 +248,58 @@ def test_vote_semantics():
     pin_vote_semantics(O)
 
 
+def pin_downlink_forms(orc):
+    """The voted vector in its two transmitted forms (Section 2.2, "Majority vote"): literal words for a
+    hand-worked vector, exhaustive round trips over every ternary vector of length 7, and vote sums that
+    add up over groups of workers and restrict to coordinate ranges (what a sharded server relies on)."""
+    # worked by hand: pairs (bit 0 = moved, bit 1 = negative), coordinate n at bits 2(n mod 16) of word n div 16
+    v = np.zeros(17, dtype=np.int8)
+    v[[1, 5, 16]] = 1
+    v[[2, 4, 15]] = -1
+    #  n=1: 01<<2 = 0x4   n=2: 11<<4 = 0x30   n=4: 11<<8 = 0x300   n=5: 01<<10 = 0x400   n=15: 11<<30 = 0xC0000000
+    assert orc.encode_vote_2bit(v).tolist() == [0xC0000734, 0x1]
+    idx, sb = orc.encode_vote_sparse(v)
+    assert idx.tolist() == [1, 2, 4, 5, 15, 16] and sb.tolist() == [0b010110]     # entries 1, 2, 4 are negative
+    assert orc.decode_vote_2bit(np.array([0xC0000734, 0x1], np.uint32), 17).tolist() == v.tolist()
+    assert orc.decode_vote_sparse(np.array([1, 2, 4, 5, 15, 16], np.uint32), np.array([0b010110], np.uint32), 17).tolist() == v.tolist()
+    assert orc.decode_vote_2bit(np.array([0b10], np.uint32), 1).tolist() == [0]     # the unused pair
+    assert orc.decode_vote_sparse(np.array([3, 99], np.uint32), np.array([0b10], np.uint32), 5).tolist() == [0, 0, 0, 1, 0]
+    for code in range(3 ** 7):                      # every ternary vector of length 7
+        t = np.array([(code // 3 ** i) % 3 - 1 for i in range(7)], dtype=np.int8)
+        assert orc.decode_vote_2bit(orc.encode_vote_2bit(t), 7).tolist() == t.tolist()
+        i, sgn = orc.encode_vote_sparse(t)
+        assert i.shape[0] == np.count_nonzero(t) and np.all(np.diff(i.astype(np.int64)) > 0)
+        assert orc.decode_vote_sparse(i, sgn, 7).tolist() == t.tolist()
+    rng = np.random.default_rng(12)
+    d, M, K = 300, 6, 40
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    g[:, ::7] = np.abs(g[:, 1::7][:, : g[:, ::7].shape[1]])
+    idx, sgn = orc.topk_sign(g, K)
+    count = orc.vote_counts(idx, sgn, M, K, d)
+    brute = np.zeros(d, dtype=np.int64)             # by definition: sum over workers of the ternary vectors
+    for m in range(M):
+        tern = np.zeros(d, dtype=np.int64)
+        tern[idx[m]] = np.where(np.signbit(g[m][idx[m]]), -1, 1)
+        brute += tern
+    assert np.array_equal(count, brute)
+    vote, _ = orc.majority_vote(idx, sgn, M, K, d)
+    assert np.array_equal(np.sign(count).astype(np.int8), vote)
+    halves = orc.vote_counts(idx[:2], sgn[:2], 2, K, d) + orc.vote_counts(idx[2:], sgn[2:], M - 2, K, d)
+    assert np.array_equal(halves, count)
+    x = rng.standard_normal(d).astype(np.float32)
+    via2 = orc.apply_vote(x, orc.decode_vote_2bit(orc.encode_vote_2bit(vote), d), 0.37)
+    vias = orc.apply_vote(x, orc.decode_vote_sparse(*orc.encode_vote_sparse(vote), d), 0.37)
+    want = orc.apply_vote(x, vote, 0.37)
+    assert np.array_equal(f32_bits(via2), f32_bits(want)) and np.array_equal(f32_bits(vias), f32_bits(want))
+    # the bit counts as Section 2.2 writes them: K + K log2(N / K), equal to N at K = N (signSGD's one bit each)
+    assert orc.uplink_bits(2 ** 10, 2 ** 20) == 2 ** 10 * 11 and orc.uplink_bits(4096, 4096) == 4096
+    assert orc.downlink_bits(2 ** 10, 2 ** 20) == 2 ** 10 * 11 and orc.uplink_bits(0, 100) == 0.0
+
+
+def test_downlink_forms():
+    pin_downlink_forms(O)
+
+
 def test_special_values_order():
     """NaN > Inf > finite > denormal > 0 in the bit-pattern order; signs taken from the sign bit."""
     g = np.array([[1.0, -np.inf, 1e-42, np.nan, -0.0, 3e38, -1e-45, 0.0]], dtype=np.float32)
@@ -565,11 +617,13 @@ def test_randk_mixer_known_answers():
 # ------------------------------------------- the pins notice planted mistakes
 ALL_PINS = [pin_bruteforce, pin_example1, pin_gamma_one_is_signsgd_mv, pin_single_worker,
             pin_invariants, pin_apply_bits, pin_vote_semantics, pin_error_feedback, pin_momentum,
-            pin_randk_subset, pin_randk_k_equals_d_is_signsgd_mv, pin_randk_uniform_and_independent]
+            pin_randk_subset, pin_randk_k_equals_d_is_signsgd_mv, pin_randk_uniform_and_independent,
+            pin_downlink_forms]
 
 
 def _mutants():
     real_topk, real_vote, real_apply = O.topk_sign, O.majority_vote, O.apply_vote
+    real_counts, real_enc2, real_encs = O.vote_counts, O.encode_vote_2bit, O.encode_vote_sparse
 
     def higher_index_wins(g, K):            # wrong tie rule
         M, d = g.shape
@@ -687,7 +741,21 @@ def _mutants():
     def randk_identity_rounds(j, d, keys):                              # no mixing: keeps the first K coordinates
         return np.asarray(j).astype(np.uint32)
 
-    extra_randk = [("randk_permutation", randk_modulo_instead_of_walk), ("randk_round_keys", randk_same_subset_for_every_worker),
+    def two_bit_msb_first(vote):                                        # pairs filled from the top of the word
+        return real_enc2(np.asarray(vote)[::-1])
+
+    def sparse_positive_is_one(vote):                                   # sign bits inverted
+        return real_encs(-np.asarray(vote, dtype=np.int8))
+
+    def counts_once_per_coordinate(idx, signbits, M, K, d):             # a coordinate counted once whoever votes
+        c = np.zeros(d, dtype=np.int64)
+        full = real_counts(idx, signbits, M, K, d)
+        c[full != 0] = np.sign(full[full != 0])
+        return c
+
+    extra_down = [("encode_vote_2bit", two_bit_msb_first), ("encode_vote_sparse", sparse_positive_is_one),
+                  ("vote_counts", counts_once_per_coordinate)]
+    extra_randk = extra_down + [("randk_permutation", randk_modulo_instead_of_walk), ("randk_round_keys", randk_same_subset_for_every_worker),
                    ("randk_round_keys", randk_same_subset_every_iteration), ("randk_permutation", randk_identity_rounds)]
     extra = extra_randk + [("error_feedback_step", ef_memory_of_raw_gradient), ("error_feedback_step", ef_kept_entries_not_cleared),
              ("error_feedback_step", ef_eta_on_gradient), ("apply_vote_momentum", momentum_uses_old_v),
@@ -698,7 +766,7 @@ def _mutants():
             ("apply_vote", apply_plus), ("apply_vote", apply_double)]
 
 
-@pytest.mark.parametrize("which", range(19))
+@pytest.mark.parametrize("which", range(22))
 def test_pins_catch_planted_mistakes(which, monkeypatch):
     name, fn = _mutants()[which]
     monkeypatch.setattr(O, name, fn)
