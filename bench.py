@@ -59,7 +59,7 @@ def byte_models(M, d, K):
     """Algorithmic bytes of one step under the four models that are reported side by side.
 
     json   4Md + message written and read + int32 vote counters (8d) + x read and written (8d): the
-           count the throughput target was stated on
+           count the throughput target was stated on (K = d: 4Md + 16d, there is no message)
     dense  the same with the vote counters this library uses in the fused step (one byte per
            coordinate up to 127 workers: 2d; int32 above: 8d)
     moved  dense without the message: the fused step without optional outputs never writes one
@@ -67,6 +67,9 @@ def byte_models(M, d, K):
     """
     words = (K + 31) // 32
     b_grad = 4 * M * d
+    if K == d:          # signSGD with majority vote: no selection, no message, no counters in memory
+        return {"grad": b_grad, "json": b_grad + 16 * d, "dense": b_grad + 8 * d, "moved": b_grad + 8 * d,
+                "min": b_grad + 8 * d}
     b_sel = 2 * M * (4 * K + 4 * words)
     b_count = 2 * d if M <= 127 else 8 * d
     return {"grad": b_grad, "json": b_grad + b_sel + 16 * d, "dense": b_grad + b_sel + b_count + 8 * d,

@@ -205,16 +205,23 @@ S3GD_API s3gd_status s3gd_last_device_status(const void* ws, void* stream);
 /*
  * Test hooks for the exactness safety net (the paper has no counterpart).
  *
- * For 0 < K <= d/4 the selection reads each gradient row once: a threshold taken at a fixed
- * rank of a 65,536-entry sample of the row filters the row, and the top K are then found
+ * For 0 < K <= d/4 the selection reads each gradient row once: a threshold tau_lo taken at a
+ * fixed rank of a 65,536-entry sample of the row filters the row, and the top K are then found
  * among the survivors.  A row whose filter kept fewer than K entries (threshold too high) or
  * more than the workspace has room for (too low) is redone exactly over the whole row; that
  * decision is taken per row on the device, and with a sound sampling rank it is almost never
- * needed.  These two calls are s3gd_topk_sign and s3gd_step with the sampling rank given by
- * the caller, so that a test can force either failure on ordinary data: sample_rank = 1 puts
- * the threshold at the largest sampled magnitude (too few survivors), a rank near 65,536 puts
- * it at the smallest (too many).  sample_rank = 0 means the library's own rank.  The results
- * must be, and are checked to be, identical to those of the ordinary calls; info[1] of
+ * needed.  The fused step without optional outputs, for K around 0.4 % of d and more, also takes
+ * a second threshold tau_hi from the sample, at a rank BELOW the expected one: entries at or
+ * above it are the largest of the row, so they vote during the filter pass itself, and only
+ * the band between the two thresholds is listed.  If more than K entries turn out to lie at or
+ * above tau_hi the row is redone too, and the votes that should not have been cast are taken back.
+ * These two calls are s3gd_topk_sign and s3gd_step with the ranks given by the caller, so that
+ * a test can force every one of these failures on ordinary data:
+ *   sample_rank   rank of tau_lo; 1 puts it at the largest sampled magnitude (too few survivors),
+ *                 a rank near 65,536 at the smallest (too many); 0 = the library's own rank
+ *   prevote_rank  rank of tau_hi; a rank well above 65,536 * K / d makes more than K entries
+ *                 vote early; 0 = the library's own rank
+ * The results must be, and are tested to be, identical to those of the ordinary calls; info[1] of
  * s3gd_device_status counts the rows that were redone.  Workspace as for the ordinary calls.
  */
 S3GD_API s3gd_status s3gd_debug_topk_sign(const float* grads, int M, uint64_t d, uint64_t K,
@@ -222,7 +229,55 @@ S3GD_API s3gd_status s3gd_debug_topk_sign(const float* grads, int M, uint64_t d,
                                           void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank);
 S3GD_API s3gd_status s3gd_debug_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr,
                                      uint32_t* opt_idx, uint32_t* opt_signbits, int8_t* opt_vote,
-                                     void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank);
+                                     void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank,
+                                     uint32_t prevote_rank);
+
+/*
+ * The step when the workers of Algorithm 1 sit on several GPUs.  The library does not communicate:
+ * these are the pieces on either side of the caller's collective.
+ *
+ * s3gd_vote_apply -- majority vote (Section 2.2 "Majority vote") over a message gathered from several
+ * senders, fused with the update (Eq. (7)); equals s3gd_majority_vote + s3gd_apply over all workers.
+ *   msg           dev, const  n_groups pieces, group_stride uint32 words apart; a piece is what one sender
+ *                             produced with s3gd_topk_sign / s3gd_randk_sign for its M_group workers:
+ *                             indices [M_group x K] directly followed by sign words [M_group x ceil(K/32)]
+ *                             (an all-gather of equal pieces has group_stride = M_group * (K + ceil(K/32)))
+ *   ws            dev         >= s3gd_workspace_bytes(n_groups * M_group, d, K)
+ *   opt_vote      dev or NULL [d] int8
+ * Contract: no worker repeats an index (true of the two producers above); with up to 127 workers the
+ * votes are then counted in bytes.  A message that may repeat indices goes to s3gd_majority_vote.
+ * An index >= d is skipped and S3GD_ERR_INDEX_RANGE recorded, as there.
+ *
+ * s3gd_vote_counts -- the sums before the sign, for a server that is split over GPUs by coordinate
+ * range: every GPU sums the votes of its own workers, the sums are added across GPUs (reduce-scatter),
+ * each GPU takes the sign of its range.  count[n] = sum over the M workers of their vote on n.
+ *   out_counts      dev  [d_padded] counts, d_padded >= d a multiple of 4 (coordinates beyond d hold zero)
+ *   bytes_per_count 4: int32 sums.  1: one byte per coordinate holding 128 + sum (M <= 127, same contract
+ *                   as above); adding R such buffers bytewise modulo 256 gives 128 * R + total, which
+ *                   s3gd_encode_vote2 undoes when told R, provided the total stays within +-127.
+ *   opt_bad_count   dev or NULL  receives the number of indices >= d that were skipped
+ *
+ * s3gd_encode_vote2 / s3gd_apply_vote2 -- the server's message in a dense form of two bits per
+ * coordinate (bit 0: moved, bit 1: negative; 0 -> 00, +1 -> 01, -1 -> 11; sixteen coordinates per uint32
+ * word, lowest bits first, padding 00), a sixteenth of the int32 sums and a quarter of the int8 vote.
+ * The paper counts |N^t| + |N^t| log2(N / |N^t|) <= N bits for this message with an index code; two
+ * bits each is the form a GPU can write and read at memory speed.
+ *   src, src_kind   dev, const  n values: kind 0 int32 sums, kind 1 bytes as written by s3gd_vote_counts
+ *                   and summed over n_summed buffers, kind 2 an int8 vote (any positive = +1, negative = -1)
+ *   out_words       dev  [ceil(n / 16)]
+ *   s3gd_apply_vote2: x[n] <- fl32(x[n] - lr * vote[n]) from the words, one rounding, unmoved bits left
+ *                   alone; opt_vote (dev or NULL, [d] int8) receives the decoded vote.
+ */
+S3GD_API s3gd_status s3gd_vote_apply(float* x, const uint32_t* msg, int n_groups, uint64_t group_stride, int M_group,
+                                     uint64_t K, uint64_t d, float lr, int8_t* opt_vote,
+                                     void* ws, size_t ws_bytes, void* stream);
+S3GD_API s3gd_status s3gd_vote_counts(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
+                                      uint64_t d_padded, void* out_counts, int bytes_per_count,
+                                      uint32_t* opt_bad_count, void* stream);
+S3GD_API s3gd_status s3gd_encode_vote2(const void* src, int src_kind, uint32_t n_summed, uint64_t n,
+                                       uint32_t* out_words, void* stream);
+S3GD_API s3gd_status s3gd_apply_vote2(float* x, const uint32_t* words, uint64_t d, float lr, int8_t* opt_vote,
+                                      void* stream);
 
 /*
  * Majority vote without any caller-provided scratch (the paper has no counterpart: this is

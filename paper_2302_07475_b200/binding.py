@@ -14,7 +14,8 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libs3gd.so")
+# S3GD_LIBRARY names another build of the same library (same C ABI) to load instead of the in-tree one
+LIB_PATH = os.environ.get("S3GD_LIBRARY") or os.path.join(_PKG, "libs3gd.so")
 
 S3GD_OK = 0
 STATUS_NAMES = {
@@ -26,7 +27,8 @@ EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd
            "s3gd_apply", "s3gd_step", "s3gd_device_status", "s3gd_profile_begin", "s3gd_profile_end",
            "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
            "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter", "s3gd_last_device_status",
-           "s3gd_debug_topk_sign", "s3gd_debug_step")
+           "s3gd_debug_topk_sign", "s3gd_debug_step", "s3gd_vote_apply", "s3gd_vote_counts", "s3gd_encode_vote2",
+           "s3gd_apply_vote2")
 
 
 class S3gdError(RuntimeError):
@@ -89,7 +91,15 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_debug_topk_sign.restype = ctypes.c_int
     lib.s3gd_debug_topk_sign.argtypes = lib.s3gd_topk_sign.argtypes + [u32]
     lib.s3gd_debug_step.restype = ctypes.c_int
-    lib.s3gd_debug_step.argtypes = lib.s3gd_step.argtypes + [u32]
+    lib.s3gd_debug_step.argtypes = lib.s3gd_step.argtypes + [u32, u32]
+    lib.s3gd_vote_apply.restype = ctypes.c_int
+    lib.s3gd_vote_apply.argtypes = [vp, u32p, ctypes.c_int, u64, ctypes.c_int, u64, u64, ctypes.c_float, vp, vp, sz, vp]
+    lib.s3gd_vote_counts.restype = ctypes.c_int
+    lib.s3gd_vote_counts.argtypes = [u32p, u32p, ctypes.c_int, u64, u64, u64, vp, ctypes.c_int, vp, vp]
+    lib.s3gd_encode_vote2.restype = ctypes.c_int
+    lib.s3gd_encode_vote2.argtypes = [vp, ctypes.c_int, u32, u64, u32p, vp]
+    lib.s3gd_apply_vote2.restype = ctypes.c_int
+    lib.s3gd_apply_vote2.argtypes = [vp, u32p, u64, ctypes.c_float, vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -213,16 +223,67 @@ def s3gd_debug_topk_sign(grads: torch.Tensor, K: int, out_idx: torch.Tensor, out
 
 def s3gd_debug_step(x: torch.Tensor, grads: torch.Tensor, K: int, lr: float, ws: torch.Tensor, sample_rank: int,
                     opt_idx: Optional[torch.Tensor] = None, opt_signbits: Optional[torch.Tensor] = None,
-                    opt_vote: Optional[torch.Tensor] = None) -> None:
-    """s3gd_step with the sampling rank of the filter threshold forced (0: the library's own)."""
+                    opt_vote: Optional[torch.Tensor] = None, prevote_rank: int = 0) -> None:
+    """s3gd_step with the sampling ranks of the two filter thresholds forced (0: the library's own)."""
     g = _ptr(grads, torch.float32, name="grads")
     M, d = grads.shape
     args = (_ptr(x, torch.float32, d, "x"), g, M, d, K, ctypes.c_float(lr),
             _ptr(opt_idx, torch.int32, M * K, "opt_idx"), _ptr(opt_signbits, torch.int32, M * words(K), "opt_signbits"),
             _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
     with torch.cuda.device(x.device):
-        code = load().s3gd_debug_step(*args, _stream(x), int(sample_rank))
+        code = load().s3gd_debug_step(*args, _stream(x), int(sample_rank), int(prevote_rank))
     _check("s3gd_debug_step", code)
+
+
+def s3gd_vote_apply(x: torch.Tensor, msg: torch.Tensor, n_groups: int, group_stride: int, M_group: int, K: int,
+                    lr: float, ws: torch.Tensor, opt_vote: Optional[torch.Tensor] = None) -> None:
+    """Vote over a message gathered from n_groups senders (each piece: indices then sign words) fused with the update."""
+    d = x.numel()
+    need = (n_groups - 1) * group_stride + M_group * (K + words(K)) if n_groups > 0 else 0
+    args = (_ptr(x, torch.float32, name="x"), _ptr(msg, torch.int32, need, "msg"), n_groups, group_stride, M_group, K, d,
+            ctypes.c_float(lr), _ptr(opt_vote, torch.int8, d, "opt_vote"), _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(x.device):
+        code = load().s3gd_vote_apply(*args, _stream(x))
+    _check("s3gd_vote_apply", code)
+
+
+def s3gd_vote_counts(idx: torch.Tensor, signbits: torch.Tensor, M: int, K: int, d: int, out_counts: torch.Tensor,
+                     opt_bad_count: Optional[torch.Tensor] = None) -> None:
+    """Vote sums of M workers into out_counts: uint8 [d_padded] (128 + sum) or int32 [d_padded] (sum)."""
+    if out_counts.dtype == torch.uint8:
+        per, p = 1, _ptr(out_counts, torch.uint8, d, "out_counts")
+    else:
+        per, p = 4, _ptr(out_counts, torch.int32, d, "out_counts")
+    args = (_ptr(idx, torch.int32, M * K, "idx"), _ptr(signbits, torch.int32, M * words(K), "signbits"), M, K, d,
+            out_counts.numel(), p, per, _ptr(opt_bad_count, torch.int32, 1, "opt_bad_count"))
+    with torch.cuda.device(out_counts.device):
+        code = load().s3gd_vote_counts(*args, _stream(out_counts))
+    _check("s3gd_vote_counts", code)
+
+
+def s3gd_encode_vote2(src: torch.Tensor, out_words: torch.Tensor, n_summed: int = 1) -> None:
+    """Two-bit form of the vote from int32 sums, from summed biased bytes (uint8) or from an int8 vote."""
+    n = src.numel()
+    if src.dtype == torch.int32:
+        kind, p = 0, _ptr(src, torch.int32, name="src")
+    elif src.dtype == torch.uint8:
+        kind, p = 1, _ptr(src, torch.uint8, name="src")
+    else:
+        kind, p = 2, _ptr(src, torch.int8, name="src")
+    args = (p, kind, n_summed, n, _ptr(out_words, torch.int32, (n + 15) // 16, "out_words"))
+    with torch.cuda.device(src.device):
+        code = load().s3gd_encode_vote2(*args, _stream(src))
+    _check("s3gd_encode_vote2", code)
+
+
+def s3gd_apply_vote2(x: torch.Tensor, words2: torch.Tensor, lr: float, opt_vote: Optional[torch.Tensor] = None) -> None:
+    """x <- x - lr * vote with the vote in its two-bit form."""
+    d = x.numel()
+    args = (_ptr(x, torch.float32, name="x"), _ptr(words2, torch.int32, (d + 15) // 16, "words"), d, ctypes.c_float(lr),
+            _ptr(opt_vote, torch.int8, d, "opt_vote"))
+    with torch.cuda.device(x.device):
+        code = load().s3gd_apply_vote2(*args, _stream(x))
+    _check("s3gd_apply_vote2", code)
 
 
 PHASES = ("sample", "filter", "threshold", "emit", "apply")

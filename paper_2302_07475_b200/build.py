@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libs3gd.so")
-SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu", "s3gd_select_small.cu", "s3gd_noalloc.cu", "s3gd_randk.cu"]
+SOURCES = ["s3gd_api.cu", "s3gd_vote.cu", "s3gd_signplane.cu", "s3gd_filter.cu", "s3gd_select.cu", "s3gd_select_small.cu", "s3gd_noalloc.cu", "s3gd_randk.cu", "s3gd_exchange.cu"]
 HEADERS = ["s3gd_common.cuh", "s3gd_tile.cuh", "s3gd_select_emit.inl"]
 
 
@@ -34,6 +34,8 @@ def _stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu file for sm_100a into one shared library; returns its path."""
+    if os.environ.get("S3GD_LIBRARY"):          # another build was asked for: leave the in-tree one alone
+        return os.environ["S3GD_LIBRARY"]
     if not force and not _stale():
         return LIB
     cmd = [

@@ -24,6 +24,7 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   L->M = M; L->d = d; L->K = K;
   L->n_tiles = (uint32_t)((d + kTileElems - 1) / kTileElems);
   L->cap = 0; L->typical_cand = 0; L->n_sample = 0; L->j_rank = 0; L->sample_stride = 0;
+  L->j_hi_rank = 0; L->dense = false;
   const bool use_filter = K > 0 && K < d && K * 4 <= d;
   if (use_filter) {
     const double p = (double)K / (double)d;
@@ -39,6 +40,10 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
       L->n_sample = (uint32_t)(chunks * 32);
       const double s = (double)L->n_sample * p;
       j = ceil(s + 6.0 * sqrt(s) + 4.0);
+      // the mirror image for the band form: with at most j_hi sampled entries at or above tau_hi, the
+      // chance that more than K entries of the row are is as small as the one above
+      const double jh = floor(s - 6.0 * sqrt(s) - 4.0);
+      L->j_hi_rank = jh >= 1.0 ? (uint32_t)jh : 0u;
     }
     if (j > (double)L->n_sample) j = (double)L->n_sample;
     if (j < 1.0) j = 1.0;
@@ -51,6 +56,7 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
     double typical = ceil(r * j * 1.25);
     if (typical > cap) typical = cap;
     L->typical_cand = (uint32_t)typical;
+    L->dense = (uint64_t)L->typical_cand * 250u > d;
   }
   size_t off = 0;
   L->off_hdr = off;      off = align_up(off + kHdrWords * sizeof(uint32_t), 256);
@@ -59,8 +65,9 @@ bool make_layout(int M, uint64_t d, uint64_t K, Layout* L) {
   L->off_seg = off;      off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
   L->off_segscan = off;  off = align_up(off + (size_t)M * L->n_tiles * sizeof(uint2), 256);
   L->off_cand = off;     off = align_up(off + (size_t)M * L->cap * sizeof(uint2), 256);
-  // bin list of the two-pass selection: at most what one CTA's shared memory takes
-  L->bin_cap = L->cap < kSmallSelectBytes / 8u ? L->cap : kSmallSelectBytes / 8u;
+  // bin list of the two-pass selection: room for a whole row's candidates, because the band form of the
+  // filter pass leaves its list unordered and has no other route for a row whose bin is long
+  L->bin_cap = L->cap;
   L->off_bin = off;      off = align_up(off + (size_t)M * L->bin_cap * sizeof(uint2), 256);
   L->off_counter = off;  off = align_up(off + (size_t)d * sizeof(int32_t), 256);
   L->total = off;
@@ -163,16 +170,17 @@ size_t s3gd_workspace_bytes(int M, uint64_t d, uint64_t K) {
 namespace {
 // sample_rank != 0 replaces the sampling plan's rank (the debug entry points); the workspace
 // layout, and with it the candidate capacity, stays that of the plan.
-void override_sample_rank(Layout* L, uint32_t sample_rank) {
-  if (sample_rank == 0u || L->cap == 0u) return;
-  L->j_rank = sample_rank < L->n_sample ? sample_rank : L->n_sample;
+void override_sample_rank(Layout* L, uint32_t sample_rank, uint32_t prevote_rank) {
+  if (L->cap == 0u) return;
+  if (sample_rank != 0u) L->j_rank = sample_rank < L->n_sample ? sample_rank : L->n_sample;
+  if (prevote_rank != 0u) L->j_hi_rank = prevote_rank < L->n_sample ? prevote_rank : L->n_sample;
 }
 
 s3gd_status topk_sign_impl(const float* grads, int M, uint64_t d, uint64_t K, uint32_t* out_idx,
                            uint32_t* out_signbits, void* ws, size_t ws_bytes, void* stream, uint32_t sample_rank) {
   Layout L;
   if (!make_layout(M, d, K, &L) || grads == nullptr || !aligned(grads, 4)) return S3GD_ERR_INVALID_ARG;
-  override_sample_rank(&L, sample_rank);
+  override_sample_rank(&L, sample_rank, 0u);
   if (K > 0 && (out_idx == nullptr || out_signbits == nullptr || !aligned(out_idx, 4) || !aligned(out_signbits, 4)))
     return S3GD_ERR_INVALID_ARG;
   s3gd_status s = check_ws(L, ws, ws_bytes);
@@ -284,10 +292,10 @@ s3gd_status check_step_args(const float* x, const float* grads, uint32_t* opt_id
 namespace {
 s3gd_status plain_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
                        uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream,
-                       uint32_t sample_rank) {
+                       uint32_t sample_rank, uint32_t prevote_rank) {
   Layout L;
   if (!make_layout(M, d, K, &L)) return S3GD_ERR_INVALID_ARG;
-  override_sample_rank(&L, sample_rank);
+  override_sample_rank(&L, sample_rank, prevote_rank);
   s3gd_status s = check_step_args(x, grads, opt_idx, opt_signbits);
   if (s != S3GD_OK) return s;
   s = check_ws(L, ws, ws_bytes);
@@ -299,13 +307,14 @@ s3gd_status plain_step(float* x, const float* grads, int M, uint64_t d, uint64_t
 
 s3gd_status s3gd_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
                       uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream) {
-  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, 0u);
+  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, 0u, 0u);
 }
 
 s3gd_status s3gd_debug_step(float* x, const float* grads, int M, uint64_t d, uint64_t K, float lr, uint32_t* opt_idx,
                             uint32_t* opt_signbits, int8_t* opt_vote, void* ws, size_t ws_bytes, void* stream,
-                            uint32_t sample_rank) {
-  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, sample_rank);
+                            uint32_t sample_rank, uint32_t prevote_rank) {
+  return plain_step(x, grads, M, d, K, lr, opt_idx, opt_signbits, opt_vote, ws, ws_bytes, stream, sample_rank,
+                    prevote_rank);
 }
 
 s3gd_status s3gd_step_ex(float* x, const float* grads, float* opt_err, float eta, float* opt_v, float mu, int M,

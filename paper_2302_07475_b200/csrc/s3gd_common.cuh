@@ -61,8 +61,13 @@ struct RowState {
   uint32_t ticket_count;  // blocks of the count pass that have finished this row
   uint32_t done;          // 0: open; 1: finished by an on-chip selection; 2, 3: taken by the two-pass form (s3gd_select.cu)
   uint32_t n_bin;         // entries collected so far in the row's bin list (two-pass form, votes only)
-  uint32_t pad[4];
+  uint32_t tau_hi;        // band form of the filter pass: entries with magnitude >= tau_hi voted during that pass
+                          // (kNoPrevote: no entry did); the candidates are then the band [tau_lo, tau_hi)
+  uint32_t n_hi;          // how many entries voted during the filter pass
+  uint32_t pad[2];
 };
+static_assert(sizeof(RowState) == 64, "one row state per 64 bytes");
+constexpr uint32_t kNoPrevote = 0x80000000u;       // above every magnitude key
 
 // Byte offsets of the workspace regions; computed identically for sizing and use.
 struct Layout {
@@ -73,8 +78,10 @@ struct Layout {
   uint32_t typical_cand; // survivors a row is expected to have (mean of the sampling plan plus grid slack)
   uint32_t n_sample;     // sampled entries per row
   uint32_t j_rank;       // sample rank that fixes tau_lo
+  uint32_t j_hi_rank;    // sample rank that fixes tau_hi in the band form (0: nothing votes during the filter pass)
   uint32_t sample_stride;  // distance between sampled groups of 8 (0: whole row sampled)
   uint32_t bin_cap;      // entries per row of the bin list (0: none)
+  bool dense;            // survivors are expected in nearly every 128-entry step of the filter pass
   size_t off_hdr, off_rows, off_hist, off_seg, off_segscan, off_cand, off_bin, off_counter, total;
 };
 
@@ -115,8 +122,11 @@ __device__ __forceinline__ uint32_t ld_stream_u32(const void* p) {
 constexpr uint32_t kRowTwoPass = 2u, kRowBin = 3u;
 
 // Does this row take its top-K from the filtered candidates (true) or from the whole row?
+// Band form: the n_hi entries at or above tau_hi have voted already.  They are the n_hi largest of
+// the row, so they belong to the top K exactly if n_hi <= K, and the other K - n_hi are then the
+// largest of the band, provided it holds that many.  (n_hi is 0 in the plain form.)
 __device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
-  return rs.exact == 0u && rs.n_cand >= K && rs.n_cand <= cap;
+  return rs.exact == 0u && rs.n_hi <= K && rs.n_cand >= K - rs.n_hi && rs.n_cand <= cap;
 }
 // Shared memory the single-CTA selection needs for a row: bit pattern and index of every
 // candidate.  Rows that fit are finished by that kernel; the others by the general passes.
@@ -166,13 +176,16 @@ cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint
                                      uint32_t* out_signbits, cudaStream_t st);
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
                                      uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
-                                     bool packed, cudaStream_t st);
-// (zero_counter != NULL: the d vote counters there, 16-byte aligned, are cleared by the sampling launch)
+                                     bool packed, bool band, cudaStream_t st);
+// (zero_counter != NULL: the d vote counters there, 16-byte aligned, are cleared by the sampling launch;
+//  band: the band form of the filter pass -- entries at or above a second sampled threshold vote into
+//  zero_counter at once and only the band between the two thresholds is listed, in no particular order)
 struct EmitOut {
   uint32_t* idx;        // [M x K] or NULL
   uint32_t* signbits;   // [M x words] or NULL (zeroed before the launch)
   int32_t* counter;     // [d] or NULL
   uint32_t packed;      // 1: the counters are bytes (see add_vote)
+  uint32_t unordered;   // 1: the candidate lists are in no particular order (band form of the filter pass)
   float* err;           // [M x d] or NULL: error memory whose kept entries are set to zero (Eq. (6))
   uint64_t d;
   uint32_t K, words;
@@ -180,8 +193,9 @@ struct EmitOut {
 cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* cand, const uint2* seg, uint32_t* hdr,
                                 const EmitOut& o, cudaStream_t st);
 // Votes only, two-pass form: one CTA per row finishes the rows marked kRowBin from their bin lists
-cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t* hdr, const EmitOut& o,
-                              cudaStream_t st);
+// (bin_cap: entries per row of the list; lists longer than one CTA's shared memory are selected from where they lie)
+cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t bin_cap, uint32_t* hdr,
+                              const EmitOut& o, cudaStream_t st);
 // Votes only, rows too large for one SM: a cluster of 2 or 4 CTAs per row (cluster_size_for; 0 = none fits)
 uint32_t cluster_size_for(uint32_t n_cand);
 cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* cand, uint32_t* hdr, const EmitOut& o,

@@ -1,0 +1,198 @@
+// The pieces of the step that sit on either side of an exchange between GPUs when the workers
+// of Algorithm 1 are spread over several of them: the vote over a message gathered from several
+// senders fused with the update, vote sums that can be added up across GPUs, and the voted
+// vector in a dense two-bit form for the way back (Section 2.2, "Majority vote": the server's
+// message is the ternary vector sgn(sum of votes)).  Nothing here communicates; the exchange
+// itself is the caller's collective between these calls.
+#include "s3gd_common.cuh"
+
+namespace s3gd {
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+inline unsigned grid_for(uint64_t items, int per_block, int max_blocks) {
+  uint64_t b = (items + per_block - 1) / per_block;
+  if (b < 1) b = 1;
+  if (b > (uint64_t)max_blocks) b = max_blocks;
+  return (unsigned)b;
+}
+
+// Votes of a message that lies in n_groups pieces (one per sender), group_stride words apart:
+// piece g has the indices of its M_group workers, [M_group x K], at idx + g * group_stride and
+// their sign words, [M_group x ceil(K/32)], at sgn + g * group_stride.  An index >= d is skipped
+// and counted.
+__global__ void __launch_bounds__(256) vote_groups_kernel(const uint32_t* __restrict__ idx,
+                                                          const uint32_t* __restrict__ sgn, uint32_t n_groups,
+                                                          uint64_t group_stride, uint32_t M_group, uint64_t K,
+                                                          uint64_t d, int32_t* __restrict__ counter, uint32_t packed,
+                                                          uint32_t* __restrict__ bad_count, uint32_t* __restrict__ status) {
+  const uint64_t words = (K + 31) / 32;
+  const uint64_t per_group = (uint64_t)M_group * K;
+  const uint64_t total = per_group * n_groups;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  uint32_t bad = 0;
+  for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    const uint64_t g = e / per_group, r = e - g * per_group;
+    const uint64_t m = r / K, j = r - m * K;
+    const uint32_t n = idx[g * group_stride + r];
+    const uint32_t neg = (sgn[g * group_stride + m * words + (j >> 5)] >> (j & 31)) & 1u;
+    if (n < d) add_vote(counter, packed, n, neg);
+    else ++bad;
+  }
+  if (bad) {
+    if (bad_count) atomicAdd(bad_count, bad);
+    if (status) atomicOr(status, (uint32_t)kFlagIndexRange);
+  }
+}
+
+// words of `value` repeated (the zero of the counters: 0, or 0x80808080 for biased bytes)
+__global__ void __launch_bounds__(256) fill_words_kernel(uint32_t* __restrict__ p, uint64_t n_words, uint32_t value) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride) p[i] = value;
+}
+
+__device__ __forceinline__ uint32_t code_of(int c) { return c > 0 ? 1u : (c < 0 ? 3u : 0u); }   // 00, 01 (+1), 11 (-1)
+
+// sixteen coordinates -> one word of two-bit codes.  kBytes: one byte per coordinate holding the
+// sum of `n_summed` biased bytes (each 128 + a partial sum), reduced modulo 256; the total then is
+// (byte - 128 * n_summed) as a signed byte.  Otherwise int32 sums (or int8 votes, kVotes).
+template <int kKind>   // 0: int32 sums, 1: biased bytes, 2: int8 votes
+__global__ void __launch_bounds__(256) encode2_kernel(const void* __restrict__ src, uint32_t bias, uint64_t n,
+                                                      uint32_t* __restrict__ out) {
+  const uint64_t n_words = (n + 15) / 16;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += stride) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+      const uint64_t i = w * 16 + q;
+      if (i >= n) break;
+      int c;
+      if (kKind == 0) c = static_cast<const int32_t*>(src)[i];
+      else if (kKind == 1) c = (int)(int8_t)(uint8_t)(static_cast<const uint8_t*>(src)[i] - bias);
+      else c = static_cast<const int8_t*>(src)[i];
+      word |= code_of(c) << (2 * q);
+    }
+    out[w] = word;
+  }
+}
+
+__device__ __forceinline__ float moved2(float x, uint32_t code, float lr) {
+  return code == 1u ? __fsub_rn(x, lr) : __fadd_rn(x, lr);      // one rounding, as s3gd_apply
+}
+
+// x <- x - lr * vote from the two-bit form: a thread takes one word = sixteen coordinates
+__global__ void __launch_bounds__(256) apply2_kernel(float* __restrict__ x, const uint32_t* __restrict__ words,
+                                                     uint64_t d, float lr, int8_t* __restrict__ opt_vote) {
+  const uint64_t n_words = (d + 15) / 16;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += stride) {
+    const uint32_t word = words[w];
+    if (word == 0u && opt_vote == nullptr) continue;
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+      const uint64_t i = w * 16 + q;
+      if (i >= d) break;
+      const uint32_t code = (word >> (2 * q)) & 3u;
+      const bool moves = (code & 1u) != 0u;                     // the pair 10 is never sent; it leaves x alone
+      if (opt_vote) opt_vote[i] = moves ? (code == 1u ? 1 : -1) : 0;
+      if (moves) x[i] = moved2(x[i], code, lr);
+    }
+  }
+}
+
+}  // namespace
+}  // namespace s3gd
+
+using namespace s3gd;
+
+extern "C" {
+
+s3gd_status s3gd_vote_apply(float* x, const uint32_t* msg, int n_groups, uint64_t group_stride, int M_group,
+                            uint64_t K, uint64_t d, float lr, int8_t* opt_vote, void* ws, size_t ws_bytes,
+                            void* stream) {
+  if (n_groups <= 0 || M_group <= 0 || (uint64_t)n_groups * (uint64_t)M_group > 65535u) return S3GD_ERR_INVALID_ARG;
+  const int M = n_groups * M_group;
+  Layout L;
+  if (!make_layout(M, d, K, &L) || x == nullptr || !aligned(x, 4)) return S3GD_ERR_INVALID_ARG;
+  const uint64_t piece = (uint64_t)M_group * (K + (K + 31) / 32);
+  if (K > 0 && (msg == nullptr || !aligned(msg, 4) || group_stride < piece)) return S3GD_ERR_INVALID_ARG;
+  if (ws == nullptr || ws_bytes < L.total || !aligned(ws, 256)) return S3GD_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = static_cast<char*>(ws);
+  uint32_t* hdr = reinterpret_cast<uint32_t*>(base + L.off_hdr);
+  int32_t* counter = reinterpret_cast<int32_t*>(base + L.off_counter);
+  // every worker votes at most once per coordinate (the message's contract), so up to 127 workers fit bytes
+  const bool packed = M <= kPackedMaxWorkers;
+  if (cudaMemsetAsync(hdr, 0, kHdrWords * sizeof(uint32_t), st) != cudaSuccess) return S3GD_ERR_CUDA;
+  const cudaError_t ez = packed ? cudaMemsetAsync(counter, 0x80, (size_t)((d + 3) / 4) * 4, st)
+                                : cudaMemsetAsync(counter, 0, (size_t)d * sizeof(int32_t), st);
+  if (ez != cudaSuccess) return S3GD_ERR_CUDA;
+  const uint64_t total = (uint64_t)M * K;
+  if (total) {
+    vote_groups_kernel<<<grid_for(total, 256, sm_count() * 16), 256, 0, st>>>(
+        msg, msg + (uint64_t)M_group * K, (uint32_t)n_groups, group_stride, (uint32_t)M_group, K, d, counter,
+        packed ? 1u : 0u, hdr + kHdrBadIndex, hdr + kHdrStatus);
+    if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+    count_launch();
+  }
+  return launch_counter_apply(counter, packed, x, d, lr, opt_vote, st) == cudaSuccess ? S3GD_OK : S3GD_ERR_CUDA;
+}
+
+s3gd_status s3gd_vote_counts(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
+                             uint64_t d_padded, void* out_counts, int bytes_per_count, uint32_t* opt_bad_count,
+                             void* stream) {
+  if (M <= 0 || M > 65535 || d == 0 || d >= (1ull << 32) || K > d || d_padded < d || d_padded % 4 != 0 ||
+      out_counts == nullptr || !aligned(out_counts, 4) || (bytes_per_count != 1 && bytes_per_count != 4))
+    return S3GD_ERR_INVALID_ARG;
+  if (bytes_per_count == 1 && M > kPackedMaxWorkers) return S3GD_ERR_INVALID_ARG;
+  if (K > 0 && (idx == nullptr || signbits == nullptr || !aligned(idx, 4) || !aligned(signbits, 4)))
+    return S3GD_ERR_INVALID_ARG;
+  if (opt_bad_count != nullptr && !aligned(opt_bad_count, 4)) return S3GD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool packed = bytes_per_count == 1;
+  const uint64_t n_words = packed ? d_padded / 4 : d_padded;
+  fill_words_kernel<<<grid_for(n_words, 256, sm_count() * 8), 256, 0, st>>>(static_cast<uint32_t*>(out_counts), n_words,
+                                                                           packed ? kPackedZero : 0u);
+  if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+  count_launch();
+  if (opt_bad_count && cudaMemsetAsync(opt_bad_count, 0, sizeof(uint32_t), st) != cudaSuccess) return S3GD_ERR_CUDA;
+  const uint64_t total = (uint64_t)M * K;
+  if (total) {
+    vote_groups_kernel<<<grid_for(total, 256, sm_count() * 16), 256, 0, st>>>(
+        idx, signbits, 1u, 0u, (uint32_t)M, K, d, static_cast<int32_t*>(out_counts), packed ? 1u : 0u, opt_bad_count,
+        nullptr);
+    if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+    count_launch();
+  }
+  return S3GD_OK;
+}
+
+s3gd_status s3gd_encode_vote2(const void* src, int src_kind, uint32_t n_summed, uint64_t n, uint32_t* out_words,
+                              void* stream) {
+  if (src == nullptr || out_words == nullptr || n == 0 || !aligned(out_words, 4) || src_kind < 0 || src_kind > 2)
+    return S3GD_ERR_INVALID_ARG;
+  if (src_kind == 0 && !aligned(src, 4)) return S3GD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const unsigned grid = grid_for((n + 15) / 16, 256, sm_count() * 8);
+  const uint32_t bias = (128u * n_summed) & 0xFFu;
+  if (src_kind == 0) encode2_kernel<0><<<grid, 256, 0, st>>>(src, 0u, n, out_words);
+  else if (src_kind == 1) encode2_kernel<1><<<grid, 256, 0, st>>>(src, bias, n, out_words);
+  else encode2_kernel<2><<<grid, 256, 0, st>>>(src, 0u, n, out_words);
+  if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+  count_launch();
+  return S3GD_OK;
+}
+
+s3gd_status s3gd_apply_vote2(float* x, const uint32_t* words, uint64_t d, float lr, int8_t* opt_vote, void* stream) {
+  if (x == nullptr || words == nullptr || d == 0 || d >= (1ull << 32) || !aligned(x, 4) || !aligned(words, 4))
+    return S3GD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  apply2_kernel<<<grid_for((d + 15) / 16, 256, sm_count() * 8), 256, 0, st>>>(x, words, d, lr, opt_vote);
+  if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+  count_launch();
+  return S3GD_OK;
+}
+
+}  // extern "C"

@@ -36,7 +36,8 @@ constexpr int kSampleUnroll = 16;
 template <bool kEF>
 __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
                                                                 RowState* __restrict__ rows, uint32_t n_sample,
-                                                                uint32_t stride, uint32_t j_rank, uint32_t K,
+                                                                uint32_t stride, uint32_t j_rank, uint32_t j_hi,
+                                                                uint32_t K,
                                                                 uint32_t* __restrict__ hdr,
                                                                 uint32_t* __restrict__ hist,
                                                                 const float* __restrict__ err, float eta, uint32_t M,
@@ -44,7 +45,6 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
                                                                 uint32_t zero_word) {
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
-  __shared__ uint32_t s_pick[2];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (blockIdx.x >= M) {                          // a clearing block; `zero` is 16-byte aligned, n_zero words
     const uint64_t n4 = n_zero / 4, nthr = (uint64_t)(gridDim.x - M) * 1024;
@@ -62,7 +62,8 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   if (tid == 0) {
     RowState rs = {};
     rs.k_rem = K;
-    rows[row] = rs;                                // tau_lo is filled in at the end
+    rs.tau_hi = kNoPrevote;
+    rows[row] = rs;                                // tau_lo (and tau_hi, if j_hi != 0) are filled in at the end
   }
   for (uint32_t b = tid; b < (uint32_t)kHistBins; b += 1024) hist[(uint64_t)row * kHistBins + b] = 0u;
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
@@ -71,6 +72,35 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
     for (uint32_t e = tid; e < n_sample; e += 1024) {
       const uint32_t b = kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e];
       atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u);
+    }
+  } else if (!kEF) {
+    // chunk c: 32 neighbours starting in [c*stride, (c+1)*stride - 32], on a 16-byte boundary so that a
+    // lane reads four of them at once; eight lanes per chunk, four chunks per warp and load
+    const uint32_t n_chunks = n_sample / kChunk;
+    const uint32_t a4 = (uint32_t)(reinterpret_cast<uintptr_t>(rowp) >> 2) & 3u;     // the row's phase within 16 bytes
+    constexpr int kVecUnroll = 8;
+    for (uint32_t c0 = warp * 4 + (lane >> 3); c0 < n_chunks; c0 += 32 * 4 * kVecUnroll) {
+      uint4 v[kVecUnroll];
+#pragma unroll
+      for (int u = 0; u < kVecUnroll; ++u) {
+        const uint32_t c = c0 + 32 * 4 * u;
+        if (c < n_chunks) {
+          // offset inside the stride: hash scaled into [0, stride - 34) by a multiply-high (no division),
+          // then up to the next position that is 16-byte aligned in memory (at most 3 further)
+          const uint64_t p = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk + 2));
+          const uint64_t pos = ((p + a4 + 3u) & ~(uint64_t)3u) - a4 + (lane & 7u) * 4u;
+          v[u] = ld_stream_v4(rowp + pos);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kVecUnroll; ++u) {
+        if (c0 + 32 * 4 * u < n_chunks) {
+          atomicAdd(&s_hist[(v[u].x & kAbsMask) >> 16], 1u);
+          atomicAdd(&s_hist[(v[u].y & kAbsMask) >> 16], 1u);
+          atomicAdd(&s_hist[(v[u].z & kAbsMask) >> 16], 1u);
+          atomicAdd(&s_hist[(v[u].w & kAbsMask) >> 16], 1u);
+        }
+      }
     }
   } else {
     const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
@@ -100,46 +130,56 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
 #pragma unroll
   for (int s = 16; s > 0; s >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, s);
   if (lane == 0) s_wsum[warp] = part;
-  if (tid == 0) { s_pick[0] = 0xFFFFFFFFu; s_pick[1] = 0u; }
   __syncthreads();
-  if (tid == 0) {
-    // highest warp range in which the count from the top reaches j_rank
-    uint32_t above = 0;
-    for (int w = 31; w >= 0; --w) {
-      if (above + s_wsum[w] >= j_rank) { s_pick[0] = (uint32_t)w; s_pick[1] = above; break; }
-      above += s_wsum[w];
-    }
-  }
-  __syncthreads();
-  const uint32_t wsel = s_pick[0];
-  if (wsel == 0xFFFFFFFFu) {                     // fewer than j_rank samples in total: keep everything
-    if (tid == 0) rows[row].tau_lo = 0u;
-    return;
-  }
-  if (warp != wsel) return;
-  // inside the chosen 1024 bins: 32 groups of 32 bins, from the top
-  uint32_t above = s_pick[1];
-  uint32_t result = 0;
-  bool found = false;
-  for (int g = 31; g >= 0 && !found; --g) {
-    uint32_t c = s_hist[wsel * 1024 + g * 32 + lane];
-    uint32_t suffix = c;                         // inclusive count of this bin and higher bins of the group
+  // Two searches for "the highest bin b such that at least `want` sampled entries lie in bins >= b":
+  // warp 0 with want = j_rank (tau_lo is that bin's lower edge), warp 1 with want = j_hi + 1 (the bin above
+  // it is the lowest one with at most j_hi sampled entries at or above its lower edge: tau_hi).
+  __shared__ uint32_t s_res[2];
+  const bool searching = warp == 0 || (warp == 1 && j_hi != 0u);
+  const uint32_t want = warp == 0 ? j_rank : j_hi + 1u;
+  uint32_t wsel = 0xFFFFFFFFu, above = 0;
+  if (searching) {
+    const uint32_t mine = s_wsum[lane];           // one 1024-bin range per lane
+    uint32_t suffix = mine;                        // entries in this range and all higher ones
 #pragma unroll
     for (int s = 1; s < 32; s <<= 1) {
-      uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
+      const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
       if (lane + s < 32) suffix += o;
     }
-    uint32_t gtot = __shfl_sync(0xFFFFFFFFu, suffix, 0);
-    if (above + gtot >= j_rank) {
-      uint32_t ok = __ballot_sync(0xFFFFFFFFu, above + suffix >= j_rank);   // lanes 0..L satisfy it
-      int top = 31 - __clz(ok);                  // highest bin of the group that still reaches j_rank
-      result = wsel * 1024 + g * 32 + (uint32_t)top;
-      found = true;
-    } else {
+    const uint32_t ok = __ballot_sync(0xFFFFFFFFu, suffix >= want);   // lanes 0..L satisfy it
+    if (ok != 0u) {
+      wsel = 31u - (uint32_t)__clz(ok);
+      above = __shfl_sync(0xFFFFFFFFu, suffix - mine, wsel);
+    }
+  }
+  uint32_t result = 0xFFFFFFFFu;                   // no such bin: fewer than `want` samples in total
+  if (searching && wsel != 0xFFFFFFFFu) {
+    // inside the chosen 1024 bins: 32 groups of 32 bins, from the top
+    for (int g = 31; g >= 0; --g) {
+      const uint32_t c = s_hist[wsel * 1024 + g * 32 + lane];
+      uint32_t suffix = c;                         // inclusive count of this bin and higher bins of the group
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
+        if (lane + s < 32) suffix += o;
+      }
+      const uint32_t gtot = __shfl_sync(0xFFFFFFFFu, suffix, 0);
+      if (above + gtot >= want) {
+        const uint32_t ok = __ballot_sync(0xFFFFFFFFu, above + suffix >= want);   // lanes 0..L satisfy it
+        result = wsel * 1024 + g * 32 + (31u - (uint32_t)__clz(ok));   // highest bin of the group that still reaches it
+        break;
+      }
       above += gtot;
     }
   }
-  if (lane == 0) rows[row].tau_lo = result << 16;
+  if (lane == 0 && warp == 0) s_res[0] = result == 0xFFFFFFFFu ? 0u : result << 16;   // too few samples: keep everything
+  // bins run to 32767, so the bin above the highest one gives 0x80000000 = kNoPrevote by itself
+  if (lane == 0 && warp == 1) s_res[1] = !searching ? kNoPrevote : (result == 0xFFFFFFFFu ? 0u : (result + 1u) << 16);
+  __syncthreads();
+  if (tid == 0) {
+    rows[row].tau_lo = s_res[0];
+    rows[row].tau_hi = s_res[1] > s_res[0] ? s_res[1] : s_res[0];      // never below tau_lo: what votes early has passed the filter
+  }
 }
 
 // Persistent CTAs over (row, tile); CTA c takes the items c, c + gridDim.x, ...  Survivors of a
@@ -433,11 +473,234 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
   }
 }
 
+
+// ---- the band form of the pass, for the fused step without outputs where survivors are dense.
+// Two thresholds come from the sample: tau_lo as above and tau_hi, placed so that (with the same
+// confidence) FEWER than K entries of the row lie at or above it.  Those entries are the largest
+// of the row, hence part of its top K whenever there are at most K of them, so they vote at once
+// and are only counted; what is listed is the band tau_lo <= magnitude < tau_hi, from which the
+// remaining K - n_hi are selected afterwards -- a fraction of what the plain form lists.  Whether
+// the guess held (n_hi <= K <= n_hi + band) is checked per row on the device after the pass; a row
+// where it did not is redone over the whole row, and the emission of that route takes back the votes
+// of entries that voted here without belonging to the top K.
+// Votes need no order, and ties at the K-th magnitude are cut by index, which every listed entry
+// carries; so the list is unordered and nothing is ranked.  The kernel is built to issue few
+// instructions per entry, because with survivors in nearly every 128-entry step the ranked forms
+// are bound by instruction issue, not by memory:
+//   A  a lane takes the largest magnitude of its four entries of a step (three max operations that
+//      keep NaN) and compares once; only a lane that has a survivor looks closer and pushes it
+//      (bit pattern, index) onto the CTA's queue with one shared-memory atomic;
+//   C  after the tile's one barrier all threads drain the queue side by side, one entry each: an
+//      entry at or above tau_hi votes, a band entry moves to the CTA's band buffer;
+//   D  one tile later the band buffer's count is final and thread 0 claims room in the row's list;
+//   F  another tile later the claim has returned and the buffer is copied out, coalesced.
+// Three buffers of each kind, so that a buffer is never refilled before its readers have passed
+// the next barrier.  Whatever does not fit a buffer is handled entry by entry at once (rare).
+
+__device__ __forceinline__ float max_keep_nan(float a, float b) {   // maximum that is NaN if either operand is
+  float r;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+
+struct BandCtx {
+  uint32_t tau_hi, packed, cap;
+  int32_t* counter;
+  uint32_t* n_cand;          // the row's list counter
+  uint2* out;                // the row's list
+};
+
+// An entry that found no room in a shared-memory buffer: vote, or claim one place in the row's list.
+// Returns 1 if it voted.
+__device__ __noinline__ uint32_t band_direct(const BandCtx c, uint32_t bits, uint32_t idx) {
+  if ((bits & kAbsMask) >= c.tau_hi) {
+    add_vote(c.counter, c.packed, idx, bits >> 31);
+    return 1u;
+  }
+  const uint32_t g = atomicAdd(c.n_cand, 1u);
+  if (g < c.cap) c.out[g] = make_uint2(bits, idx);
+  return 0u;
+}
+
+// Push onto the CTA's queue.  An entry that finds the queue full lands in the spare slot behind it;
+// the count keeps running, and a tile that pushed more than the queue holds is redone entry by entry.
+__device__ __forceinline__ void queue_push(uint2* q, uint32_t* q_cnt, uint32_t bits, uint32_t idx) {
+  const uint32_t slot = atomicAdd(q_cnt, 1u);
+  q[min(slot, 4u * blockDim.x)] = make_uint2(bits, idx);      // (the queue holds 4 entries per thread)
+}
+
+// The first tile of a row whose start is not on a 128-byte boundary, the ragged last tile, and
+// (direct) any tile that pushed more than the queue holds: every entry is loaded and tested by
+// itself and either pushed or, in the direct form, handled at once.  e0: row index of the thread's
+// first entry of the tile (its others follow in steps of 128, four at a time); head: entries of the
+// row before its first 128-byte boundary, which belong to tile 0.  Returns the number of entries that voted.
+__device__ __noinline__ uint32_t band_tile_slow(const uint32_t* __restrict__ rowp, uint64_t d, uint32_t head, bool first,
+                                                uint32_t e0, float tau, uint2* q, uint32_t* q_cnt, const BandCtx c,
+                                                bool direct) {
+  uint32_t voted = 0;
+  auto take = [&](uint32_t e) {
+    const uint32_t bits = ld_stream_u32(rowp + e);
+    if (!hit(bits, tau)) return;
+    if (direct) voted += band_direct(c, bits, e);
+    else queue_push(q, q_cnt, bits, e);
+  };
+  if (first && threadIdx.x < head) take(threadIdx.x);
+#pragma unroll 1
+  for (int it = 0; it < kTileIters; ++it) {
+#pragma unroll 1
+    for (uint32_t k = 0; k < 4; ++k) {
+      const uint64_t e = (uint64_t)e0 + (uint32_t)it * 128u + k;
+      if (e < d) take((uint32_t)e);
+    }
+  }
+  return voted;
+}
+
+// kThreads threads take tiles of 32 * kThreads entries (a warp owns 1024 contiguous ones, as in the
+// other forms).  Smaller CTAs, more of them per SM: fewer warps wait on each other at the tile's barrier.
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads) filter_band_kernel(const uint32_t* __restrict__ gbits, int M,
+                                                                                uint64_t d, RowState* __restrict__ rows,
+                                                                                uint2* __restrict__ cand, uint32_t cap,
+                                                                                int32_t* __restrict__ counter,
+                                                                                uint32_t packed) {
+  constexpr uint32_t kElems = (uint32_t)kThreads * 32u;          // entries per tile
+  constexpr int kQueueCap = 4 * kThreads;                        // survivors of a tile the queue holds
+  constexpr int kBandStage = 2 * kThreads;                       // band entries of a tile the band buffer holds
+  const uint32_t n_tiles = (uint32_t)((d + kElems - 1) / kElems);
+  __shared__ uint2 s_q[3][kQueueCap + 1];            // + the spare slot that takes pushes beyond the capacity
+  __shared__ uint2 s_b[3][kBandStage];
+  __shared__ uint32_t s_qcnt[3], s_bcnt[3], s_hi[3], s_base[3];
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint64_t n_work = (uint64_t)M * n_tiles;
+  if (tid < 3) { s_qcnt[tid] = 0u; s_bcnt[tid] = 0u; s_hi[tid] = 0u; }
+  __syncthreads();
+  // tiles of this CTA, and two more rounds to let the last two tiles through steps D and F
+  const uint64_t n_mine = blockIdx.x < n_work ? (n_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  uint32_t row = (uint32_t)(blockIdx.x / n_tiles), t = (uint32_t)(blockIdx.x - (uint64_t)row * n_tiles);
+  uint32_t loaded_row = 0xFFFFFFFFu, tau_hi = kNoPrevote, e0 = 0;
+  float tau = 0.f;
+  bool fast = false;                               // the tile in flight is whole and starts on a 128-byte boundary
+  uint4 v[kTileIters];
+  auto issue_loads = [&]() {
+    const uint32_t* rowp = gbits + (uint64_t)row * d;
+    const uint32_t head = row_head(rowp, d);
+    if (row != loaded_row) {
+      loaded_row = row;
+      tau = __uint_as_float(rows[row].tau_lo);
+      tau_hi = rows[row].tau_hi;
+    }
+    fast = (uint64_t)head + (uint64_t)(t + 1) * kElems <= d && !(t == 0 && head != 0u);
+    e0 = head + t * kElems + warp * 1024u + lane * 4u;
+    if (fast) {
+      const uint32_t* p = rowp + e0;
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it) v[it] = ld_stream_v4(p + it * 128);
+    }
+  };
+  auto ctx_of = [&](uint32_t r, uint32_t th) {
+    BandCtx c;
+    c.tau_hi = th; c.packed = packed; c.cap = cap; c.counter = counter;
+    c.n_cand = &rows[r].n_cand; c.out = cand + (uint64_t)r * cap;
+    return c;
+  };
+  uint32_t row1 = 0;                               // tile k-1: its band buffer fills until this round's barrier
+  bool have1 = false;
+  uint32_t n2 = 0, row2 = 0, base2 = 0;            // tile k-2: claimed (thread 0 holds base2), copied out this round
+  int cur = 0;                                     // k % 3
+  for (uint64_t k = 0; k < n_mine + 2; ++k, cur = cur == 2 ? 0 : cur + 1) {
+    const int p1 = cur == 0 ? 2 : cur - 1, p2 = cur == 2 ? 0 : cur + 1;      // (k-1) % 3, (k-2) % 3
+    const bool live = k < n_mine;
+    if (live) {
+      if (k) next_tile(row, t, n_tiles);
+      issue_loads();
+    }
+    // tile k's identity, for the steps after the barrier
+    const uint32_t row_c = row, t_c = t, tau_hi_c = tau_hi, e0_c = e0;
+    const float tau_c = tau;
+    if (live) {
+      // ---- A: survivors of this tile -> queue
+      if (fast) {
+#pragma unroll
+        for (int it = 0; it < kTileIters; ++it) {
+          const float a = max_keep_nan(fabsf(__uint_as_float(v[it].x)), fabsf(__uint_as_float(v[it].y)));
+          const float b = max_keep_nan(fabsf(__uint_as_float(v[it].z)), fabsf(__uint_as_float(v[it].w)));
+          // a branch the whole warp takes together (no divergence to manage)
+          if (__any_sync(0xFFFFFFFFu, !(max_keep_nan(a, b) < tau))) {
+            const uint32_t idx = e0 + it * 128;
+            if (hit(v[it].x, tau)) queue_push(s_q[cur], &s_qcnt[cur], v[it].x, idx);
+            if (hit(v[it].y, tau)) queue_push(s_q[cur], &s_qcnt[cur], v[it].y, idx + 1);
+            if (hit(v[it].z, tau)) queue_push(s_q[cur], &s_qcnt[cur], v[it].z, idx + 2);
+            if (hit(v[it].w, tau)) queue_push(s_q[cur], &s_qcnt[cur], v[it].w, idx + 3);
+          }
+        }
+      } else {
+        const uint32_t* rowp = gbits + (uint64_t)row * d;
+        band_tile_slow(rowp, d, row_head(rowp, d), t == 0, e0, tau, s_q[cur], &s_qcnt[cur], ctx_of(row, tau_hi), false);
+      }
+    }
+    // ---- E: the claim made for tile k-2 a round ago has had a tile's time to return
+    if (tid == 0 && n2) s_base[p2] = base2;
+    __syncthreads();
+    // ---- F: copy out the band entries of tile k-2
+    if (n2) {
+      const uint32_t base = s_base[p2];
+      uint2* out = cand + (uint64_t)row2 * cap;
+      for (uint32_t i = tid; i < n2; i += kThreads)
+        if (base + i < cap) out[base + i] = s_b[p2][i];
+    }
+    // ---- C: drain this tile's queue, one entry per thread and round
+    if (live) {
+      uint32_t my_hi = 0;
+      const uint32_t pushed = s_qcnt[cur];
+      uint32_t n = pushed;
+      if (pushed > (uint32_t)kQueueCap) {          // (the same for every thread) more survivors than the queue holds:
+        n = 0;                                     // drop it and handle the tile's entries one by one
+        const uint32_t* rowp = gbits + (uint64_t)row_c * d;
+        my_hi = band_tile_slow(rowp, d, row_head(rowp, d), t_c == 0, e0_c, tau_c, s_q[cur], &s_qcnt[cur],
+                               ctx_of(row_c, tau_hi_c), true);
+      }
+      for (uint32_t i = tid; i < n; i += kThreads) {
+        const uint2 e = s_q[cur][i];
+        if ((e.x & kAbsMask) >= tau_hi_c) {
+          add_vote(counter, packed, e.y, e.x >> 31);
+          ++my_hi;
+        } else {
+          const uint32_t pos = atomicAdd(&s_bcnt[cur], 1u);
+          if (pos < (uint32_t)kBandStage) s_b[cur][pos] = e;
+          else band_direct(ctx_of(row_c, tau_hi_c), e.x, e.y);
+        }
+      }
+      my_hi = __reduce_add_sync(0xFFFFFFFFu, my_hi);
+      if (lane == 0 && my_hi) atomicAdd(&s_hi[cur], my_hi);
+    }
+    // ---- D: tile k-1's band buffer and vote count became final at this round's barrier
+    uint32_t n1_final = 0;
+    if (have1) {
+      const uint32_t c = s_bcnt[p1];
+      n1_final = c < (uint32_t)kBandStage ? c : (uint32_t)kBandStage;
+    }
+    uint32_t base1 = 0;
+    if (tid == 0) {
+      if (n1_final) base1 = atomicAdd(&rows[row1].n_cand, n1_final);
+      if (have1 && s_hi[p1]) atomicAdd(&rows[row1].n_hi, s_hi[p1]);
+      // buffers whose readers are all past this round's barrier: the queue of tile k-1 (drained a round
+      // ago), the band buffer and vote count of tile k-2 (claimed a round ago, copied out by threads that
+      // reach the next barrier before anyone refills it)
+      s_qcnt[p1] = 0u;
+      s_hi[p2] = 0u;
+      s_bcnt[p2] = 0u;
+    }
+    n2 = n1_final; row2 = row1; base2 = base1;
+    have1 = live; row1 = row_c;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, RowState* rows, uint2* cand, uint2* seg,
                                      uint32_t* hdr, uint32_t* hist, float* ef_err, float eta, int32_t* zero_counter,
-                                     bool packed, cudaStream_t st) {
+                                     bool packed, bool band, cudaStream_t st) {
   // ef_err != NULL: gbits are the raw gradients g~, ef_err holds e and leaves holding g = g~ + eta * e
   // 128 KB of dynamic shared memory needs the opt-in on every device this runs on
   const size_t smem = (size_t)kSampleBins * sizeof(uint32_t);
@@ -453,7 +716,8 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
     if (n_clear < 32u) n_clear += (unsigned)sm_count();
   }
   sample<<<(unsigned)L.M + n_clear, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
-                                                      (uint32_t)L.K, hdr, hist, ef_err, eta, (uint32_t)L.M, zero_counter,
+                                                      band ? L.j_hi_rank : 0u, (uint32_t)L.K, hdr, hist, ef_err, eta,
+                                                      (uint32_t)L.M, zero_counter,
                                                       packed ? (L.d + 3) / 4 : L.d, packed ? kPackedZero : 0u);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -461,7 +725,15 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   count_launch(2);
   const uint64_t n_work = (uint64_t)L.M * L.n_tiles;
   const uint64_t blocks = n_work < (uint64_t)sm_count() * 8 ? n_work : (uint64_t)sm_count() * 8;
-  const bool dense = (uint64_t)L.typical_cand * 250u > L.d;
+  if (band) {                                    // (the caller asks for it only without error memory and with counters)
+    constexpr int kBandThreads = 256;
+    const uint64_t tiles = (uint64_t)L.M * ((L.d + kBandThreads * 32 - 1) / (kBandThreads * 32));
+    const uint64_t resident = (uint64_t)sm_count() * (1024 / kBandThreads);
+    filter_band_kernel<kBandThreads><<<(unsigned)(tiles < resident ? tiles : resident), kBandThreads, 0, st>>>(
+        gbits, L.M, L.d, rows, cand, L.cap, zero_counter, packed ? 1u : 0u);
+    return cudaGetLastError();
+  }
+  const bool dense = L.dense;
   auto filter = dense ? (ef_err ? filter_scan_kernel<true> : filter_scan_kernel<false>)
                       : (ef_err ? filter_kernel<true> : filter_kernel<false>);
   filter<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles, ef_err, eta);

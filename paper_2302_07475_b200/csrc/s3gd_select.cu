@@ -31,6 +31,7 @@ __global__ void init_kernel(uint32_t* __restrict__ hdr, RowState* __restrict__ r
     RowState rs = {};
     rs.k_rem = K;
     rs.exact = force_exact;
+    rs.tau_hi = kNoPrevote;
     rows[m] = rs;
   }
   for (uint64_t i = tid; i < (uint64_t)M * kHistBins; i += nthr) hist[i] = 0u;
@@ -46,8 +47,10 @@ __device__ __forceinline__ RowState load_row_state(const RowState* p) {
   RowState rs = {};
   rs.tau_lo = p->tau_lo;
   rs.n_cand = p->n_cand;
-  rs.exact = p->exact;
   rs.done = p->done;
+  rs.tau_hi = p->tau_hi;
+  rs.n_hi = p->n_hi;
+  rs.exact = __ldcg(&p->exact);              // the first pass of the two-pass form may set it
   rs.prefix = __ldcg(&p->prefix);
   rs.k_rem = __ldcg(&p->k_rem);
   rs.tau = __ldcg(&p->tau);
@@ -120,7 +123,7 @@ __device__ __forceinline__ uint32_t joint_digit(uint32_t key, uint32_t tau_lo) {
 // histogram for the next pass.  One block of kSelThreads threads.
 __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t row, uint32_t* __restrict__ h,
                                            uint32_t* __restrict__ hdr, int pass, uint32_t* s_sum, uint32_t* s_sel,
-                                           bool joint = false, uint32_t bin_limit = 0u) {
+                                           bool joint = false, uint32_t bin_limit = 0u, bool band = false) {
   const uint32_t tid = threadIdx.x;
   const int nbins = 1 << pass_bits(pass);
   const int per = nbins / kSelThreads;               // 8 or 4 bins per thread, ascending
@@ -134,7 +137,8 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
   s_sum[tid] = mine;
   if (tid == 0) { s_sel[0] = 0xFFFFFFFFu; s_sel[1] = 0u; }
   __syncthreads();
-  const uint32_t k_rem = __ldcg(&rows[row].k_rem);
+  // (first pass of the two-pass form: whatever voted during the filter pass is no longer looked for)
+  const uint32_t k_rem = __ldcg(&rows[row].k_rem) - (joint ? rows[row].n_hi : 0u);
   uint32_t above = 0;                                // entries in bins owned by higher threads
   for (int t = kSelThreads - 1; t > (int)tid; --t) above += s_sum[t];
   if (above < k_rem && above + mine >= k_rem) {      // exactly one thread
@@ -156,6 +160,8 @@ __device__ __forceinline__ void pick_digit(RowState* __restrict__ rows, uint32_t
       rows[row].k_rem = k_rem - a;
       rows[row].done = s_sel[2] <= bin_limit ? kRowBin : kRowTwoPass;
       atomicAdd(hdr + kHdrRowsDone, 1u);
+    } else if (band) {
+      rows[row].exact = 1u;       // an unordered list cannot go through count and emission: redo the whole row
     }
   } else if (tid == 0) {
     uint32_t digit = s_sel[0], a = s_sel[1];
@@ -301,7 +307,7 @@ __device__ __forceinline__ void hist_two_pass_block(const uint2* __restrict__ ca
                                                     RowState* __restrict__ rows, uint32_t K,
                                                     uint32_t* __restrict__ hist, uint32_t* __restrict__ hdr, int pass,
                                                     uint32_t bx, uint32_t row, uint32_t gx, uint2* __restrict__ bin,
-                                                    uint32_t bin_cap, const EmitOut& o) {
+                                                    uint32_t bin_cap, const EmitOut& o, bool band) {
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_sum[kSelThreads];
   __shared__ uint32_t s_sel[3];
@@ -343,7 +349,8 @@ __device__ __forceinline__ void hist_two_pass_block(const uint2* __restrict__ ca
     }
   }
   if (last_block_of_row(&rows[row].ticket_hist, gx, &s_flag))
-    pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel, joint, o.counter != nullptr && o.idx == nullptr ? bin_cap : 0u);
+    pick_digit(rows, row, g_hist, hdr, pass, s_sum, s_sel, joint, o.counter != nullptr && o.idx == nullptr ? bin_cap : 0u,
+               band);
 }
 
 }  // namespace

@@ -274,6 +274,22 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
       self[it] = s;
     }
     const bool head_sel = T.head_valid && (hkey > rs.tau || (head_eq && sc.y + Re.head_rank < rs.take_ties));
+    // Band form of the filter pass: every entry at or above tau_hi has voted there already.  This route
+    // is the one that redoes such a row, so the kept ones among them do not vote again and the others
+    // take their vote back (an opposite vote; the counters are sums).
+    const bool prevoted = o.counter != nullptr && rs.tau_hi != kNoPrevote;     // the same for the whole row
+    if (prevoted) {
+      if (T.head_valid && hkey >= rs.tau_hi && !head_sel) add_vote(o.counter, o.packed, lane, (T.head_bits >> 31) ^ 1u);
+#pragma unroll
+      for (int it = 0; it < kTileIters; ++it) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t b = T.bits[it][q];
+          if ((T.valid[it] >> q & 1u) && (b & kAbsMask) >= rs.tau_hi && !(self[it] >> q & 1u))
+            add_vote(o.counter, o.packed, (uint32_t)(T.first(it) + q), (b >> 31) ^ 1u);
+        }
+      }
+    }
     TileRanks Rs;
     tile_ranks(Rs, self, head_sel, s_wtot);
     if (Rs.tile_total == 0) continue;
@@ -282,7 +298,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
       const uint32_t neg = T.head_bits >> 31;
       if (pos < o.K) {
         if (o.idx) o.idx[(uint64_t)row * o.K + pos] = lane;
-        if (o.counter) add_vote(o.counter, o.packed, lane, neg);
+        if (o.counter && !(prevoted && hkey >= rs.tau_hi)) add_vote(o.counter, o.packed, lane, neg);
         if (o.err) o.err[(uint64_t)row * o.d + lane] = 0.f;
         if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
       }
@@ -301,7 +317,7 @@ __device__ __forceinline__ void emit_row(const uint32_t* __restrict__ gbits, uin
             const uint32_t n = (uint32_t)(T.first(it) + q);
             const uint32_t neg = T.bits[it][q] >> 31;
             if (o.idx) o.idx[(uint64_t)row * o.K + pos] = n;
-            if (o.counter) add_vote(o.counter, o.packed, n, neg);
+            if (o.counter && !(prevoted && (T.bits[it][q] & kAbsMask) >= rs.tau_hi)) add_vote(o.counter, o.packed, n, neg);
             if (o.err) o.err[(uint64_t)row * o.d + n] = 0.f;
             const uint32_t rel = (pos >> 5) - (p0 >> 5);      // 0..4: at most 128 entries per warp-iteration
 #pragma unroll
@@ -365,8 +381,8 @@ __global__ void __launch_bounds__(kSelThreads, 6) hist_two_pass_kernel(const uin
                                                                        uint32_t* __restrict__ hist,
                                                                        uint32_t* __restrict__ hdr, int pass,
                                                                        uint2* __restrict__ bin, uint32_t bin_cap,
-                                                                       EmitOut o) {
-  hist_two_pass_block(cand, cap, rows, K, hist, hdr, pass, blockIdx.x, blockIdx.y, gridDim.x, bin, bin_cap, o);
+                                                                       EmitOut o, bool band) {
+  hist_two_pass_block(cand, cap, rows, K, hist, hdr, pass, blockIdx.x, blockIdx.y, gridDim.x, bin, bin_cap, o, band);
 }
 
 __global__ void __launch_bounds__(kSelThreads, 5) emit_kernel(const uint32_t* __restrict__ gbits, uint64_t d,
@@ -457,20 +473,9 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     count_launch();                                 \
   } while (0)
 
-  if (use_filter) {
-    cudaError_t e = ef_raw ? launch_sample_and_filter(reinterpret_cast<const uint32_t*>(ef_raw), L, rows, cand, seg,
-                                                      hdr, hist, err_to_clear, eta, counter, packed, st)
-                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, packed, st);
-    if (e != cudaSuccess) return e;
-  } else {
-    init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, sm_count() * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
-    S3GD_CHECK_LAUNCH();
-    prof_mark(kPhaseSampled, st);
-  }
-  prof_mark(kPhaseFiltered, st);
   EmitOut o;
   o.idx = out_idx; o.signbits = out_signbits; o.counter = counter; o.packed = packed ? 1u : 0u;
-  o.err = err_to_clear; o.d = L.d;
+  o.err = err_to_clear; o.d = L.d; o.unordered = 0u;
   o.K = K; o.words = (uint32_t)((L.K + 31) / 32);
   // Rows whose candidates fit one SM are finished by one CTA each; if only the votes are wanted and a
   // typical row needs the shared memory of up to four SMs, by a cluster of CTAs each.
@@ -483,16 +488,43 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     if (!fits_single_cta(expect)) cluster = cluster_size_for(expect);
     if (cluster == 0u && !fits_single_cta(L.typical_cand)) cluster = cluster_size_for(L.typical_cand);
   }
+  // If a row's candidates are expected to fit an on-chip selection, the general passes only serve the
+  // odd row that did not fit or fell back to the whole-row route.
+  const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);
+  // With error compensation rows do run past the estimate (measured: the single launch then took
+  // 1.07 ms where the five launches take 0.17 ms), so that mode keeps the five launches.
+  // Where the general passes carry the selection of candidate rows, those rows take the two-pass form
+  // first (two histogram launches instead of three, candidate blocks only); the single launch after it
+  // does whatever is left -- rows on the whole-row route, rows whose K-th magnitude lies more than a
+  // quarter octave above tau_lo -- and otherwise returns at once.
+  const bool two_pass = use_filter && !only_fallback && err_to_clear == nullptr;
+  // Only the votes wanted: the band form of the filter pass (s3gd_filter.cu), whose lists are unordered.
+  // Every selection that follows either needs no order (the on-chip ones, the bin route of the two-pass
+  // form) or sends the row to the whole-row route.
+  const bool band = use_filter && votes_only && err_to_clear == nullptr;
+  // (a row too long for the on-chip selection still has the two-pass form to go to, if that follows)
+  o.unordered = band && only_fallback ? 1u : 0u;
+
+  if (use_filter) {
+    cudaError_t e = ef_raw ? launch_sample_and_filter(reinterpret_cast<const uint32_t*>(ef_raw), L, rows, cand, seg,
+                                                      hdr, hist, err_to_clear, eta, counter, packed, false, st)
+                           : launch_sample_and_filter(gbits, L, rows, cand, seg, hdr, hist, nullptr, 0.f, counter, packed,
+                                                      band, st);
+    if (e != cudaSuccess) return e;
+  } else {
+    init_kernel<<<clampu(((uint64_t)M * kHistBins + 255) / 256, 1, sm_count() * 4), 256, 0, st>>>(hdr, rows, hist, M, K, 1u);
+    S3GD_CHECK_LAUNCH();
+    prof_mark(kPhaseSampled, st);
+  }
+  prof_mark(kPhaseFiltered, st);
   if (use_filter && (cluster != 0u || fits_single_cta(K))) {    // a candidate row has at least K candidates
     cudaError_t e = cluster ? launch_select_cluster(L, rows, cand, hdr, o, cluster, st)
                             : launch_select_small(L, rows, cand, seg, hdr, o, st);
     if (e != cudaSuccess) return e;
   }
-  // Blocks per row (each block strides over its row's candidates or tiles).  If a row's
-  // candidates are expected to fit the single-CTA selection, these launches only serve the
-  // odd row that did not fit or fell back to the whole-row route, and normally exit at once:
-  // keep them small.  Otherwise they carry the selection of all rows: about eight CTAs per SM.
-  const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);
+  // Blocks per row (each block strides over its row's candidates or tiles).  Launches that only
+  // serve the odd row normally exit at once: keep them small.  Otherwise they carry the selection
+  // of all rows: about eight CTAs per SM.
   const uint32_t per_row = (uint32_t)(((uint64_t)sm_count() * (only_fallback ? 4 : 8) + M - 1) / M);
   const uint32_t gx_hist_c = use_filter ? clampu(((uint64_t)L.cap + 4095) / 4096, 1, only_fallback ? per_row : 64) : 0u;
   // the sweeps of the two-pass form: all rows' blocks resident at once (six per SM), each with a longer
@@ -501,32 +533,27 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   const uint32_t gx_two = clampu(((uint64_t)L.cap + 4095) / 4096, 1, clampu((uint64_t)sm_count() * 6 / M, 8, 64));
   const uint32_t gx_tile_c = use_filter ? clampu(((uint64_t)L.n_tiles + 7) / 8, 1, per_row) : 0u;
   const uint32_t gx_r = clampu(L.n_tiles, 1, per_row);
-  // With error compensation rows do run past the estimate (measured: the single launch then took
-  // 1.07 ms where the five launches take 0.17 ms), so that mode keeps the five launches.
-  // Where the general passes carry the selection of candidate rows, those rows take the two-pass form
-  // first (two histogram launches instead of three, candidate blocks only); the single launch after it
-  // does whatever is left -- rows on the whole-row route, rows whose K-th magnitude lies more than a
-  // quarter octave above tau_lo -- and otherwise returns at once.
-  const bool two_pass = use_filter && !only_fallback && err_to_clear == nullptr;
   if (two_pass) {
     // bin lists only where the votes alone are wanted (the message needs positions)
     uint2* bin = reinterpret_cast<uint2*>(base + L.off_bin);
-    const uint32_t bin_cap = votes_only ? L.bin_cap : 0u;
-    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 0, bin, bin_cap, o);
+    const uint32_t bin_cap = band ? L.bin_cap : 0u;
+    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 0, bin, bin_cap, o, band);
     S3GD_CHECK_LAUNCH();
-    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 2, bin, bin_cap, o);
+    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 2, bin, bin_cap, o, band);
     S3GD_CHECK_LAUNCH();
     prof_mark(kPhaseThreshold, st);
     if (bin_cap) {
-      cudaError_t e = launch_select_bin(L, rows, bin, hdr, o, st);
+      cudaError_t e = launch_select_bin(L, rows, bin, bin_cap, hdr, o, st);
       if (e != cudaSuccess) return e;
     }
-    count_scan_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows, K, cnt,
-                                                                  hdr, gx_tile_c, kRowTwoPass);
-    S3GD_CHECK_LAUNCH();
-    emit_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
-                                                            gx_tile_c, kRowTwoPass);
-    S3GD_CHECK_LAUNCH();
+    if (!band) {                  // (the band form's lists are unordered: every row's bin goes to the bin selection)
+      count_scan_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, rows, K, cnt,
+                                                                    hdr, gx_tile_c, kRowTwoPass);
+      S3GD_CHECK_LAUNCH();
+      emit_kernel<<<dim3(gx_tile_c, M), kSelThreads, 0, st>>>(gbits, L.d, L.n_tiles, cand, L.cap, seg, cnt, rows, o,
+                                                              gx_tile_c, kRowTwoPass);
+      S3GD_CHECK_LAUNCH();
+    }
   }
   if ((only_fallback || two_pass) && err_to_clear == nullptr) {
     // as many blocks as can be resident together, and no more than the largest pass has virtual blocks

@@ -42,6 +42,159 @@ __device__ __forceinline__ uint32_t block_scan_excl_1024(uint32_t v, uint32_t* s
   return woff + inc - v;
 }
 
+
+// ---- a bin list too long for shared memory (votes only, band form of the filter pass): the same
+// decisions taken over the list where it lies, in L2 / device memory, by the row's one CTA.  The
+// entries share their upper 21 magnitude bits; one sweep counts the low 10, and if the entries
+// equal to the K-th magnitude are not all kept, three more sweeps find the index up to which they
+// are (a radix select on the index: the lowest indices win).  A last sweep lets the kept ones vote.
+// Rare for smooth data (a bin is 1024 keys wide); the rule for coarsely quantised gradients with
+// tens of thousands of equal magnitudes at the threshold.
+__device__ __forceinline__ void warp_hist_add(uint32_t* s_hist, bool on, uint32_t digit) {
+  const uint32_t act = __ballot_sync(0xFFFFFFFFu, on);
+  if (act == 0u) return;                             // warp-uniform
+  const uint32_t lead = (uint32_t)__ffs((int)act) - 1u;
+  const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, digit, lead);
+  if (__all_sync(0xFFFFFFFFu, !on || digit == d0)) {   // equal magnitudes: one add for the warp
+    if ((threadIdx.x & 31u) == lead) atomicAdd(&s_hist[d0], (uint32_t)__popc(act));
+  } else if (on) {
+    atomicAdd(&s_hist[digit], 1u);
+  }
+}
+
+// The bin among `nbins` (a power of two, at most 2048) that holds the want-th entry counted from the
+// top (descending) or from the bottom; *before = entries in the bins passed on the way.  Block-wide.
+__device__ __forceinline__ uint32_t pick_bin_1024(const uint32_t* s_hist, int nbins, bool from_top, uint32_t want,
+                                                  uint32_t* before, uint32_t* s_warp, uint32_t* s_sel) {
+  const uint32_t tid = threadIdx.x;
+  const int per = nbins > kSmallThreads ? nbins / kSmallThreads : 1;
+  uint32_t mine = 0, cbin[2] = {0u, 0u};
+  if ((int)tid * per < nbins) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      if (i < per) {
+        const int pos = (int)tid * per + i;
+        cbin[i] = s_hist[from_top ? nbins - 1 - pos : pos];
+        mine += cbin[i];
+      }
+  }
+  uint32_t total;
+  const uint32_t earlier = block_scan_excl_1024(mine, s_warp, &total);
+  if (tid == 0) s_sel[0] = 0xFFFFFFFFu;
+  __syncthreads();
+  if (earlier < want && earlier + mine >= want) {              // exactly one thread
+    uint32_t a = earlier;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      if (i < per) {
+        if (a + cbin[i] >= want) {
+          const int pos = (int)tid * per + i;
+          s_sel[0] = (uint32_t)(from_top ? nbins - 1 - pos : pos);
+          s_sel[1] = a;
+          break;
+        }
+        a += cbin[i];
+      }
+    }
+  }
+  __syncthreads();
+  *before = s_sel[1];
+  return s_sel[0];                                             // 0xFFFFFFFF: fewer than `want` entries
+}
+
+__device__ __forceinline__ void select_bin_in_place(RowState* __restrict__ rows, uint32_t row, const RowState& rs,
+                                                    const uint2* __restrict__ c, uint32_t n, uint32_t* __restrict__ hdr,
+                                                    const EmitOut& o, uint32_t* s_hist, uint32_t* s_warp,
+                                                    uint32_t* s_sel, bool overflowed) {
+  const uint32_t tid = threadIdx.x;
+  constexpr int kLoads = 4;                                    // list entries a thread has in flight
+  const uint32_t k_want = rs.k_rem;
+  bool bad = overflowed;
+  // ---- low 10 bits of the magnitude
+  for (int b = tid; b < 1024; b += kSmallThreads) s_hist[b] = 0u;
+  __syncthreads();
+  for (uint32_t base = 0; base < n; base += kSmallThreads * kLoads) {
+    uint32_t key[kLoads];
+    bool on[kLoads];
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const uint32_t i = base + u * kSmallThreads + tid;
+      on[u] = i < n;
+      key[u] = on[u] ? (c[i].x & kAbsMask) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) warp_hist_add(s_hist, on[u], key[u] & 1023u);
+  }
+  __syncthreads();
+  uint32_t above = 0;
+  uint32_t digit = pick_bin_1024(s_hist, 1024, true, k_want, &above, s_warp, s_sel);
+  if (digit == 0xFFFFFFFFu) { bad = true; digit = 0u; above = 0u; }     // cannot happen for a valid row
+  const uint32_t tau = (rs.prefix << pass_bits(kNumPasses - 1)) | digit, take = k_want - above;
+  const uint32_t n_equal = s_hist[digit];
+  __syncthreads();
+  // ---- entries equal to tau: all kept, or those with the `take` lowest indices
+  uint32_t idx_limit = 0xFFFFFFFFu;
+  if (n_equal > take) {
+    uint32_t iprefix = 0, t_rem = take;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const int prev_shift = pass == 1 ? 21 : 10;
+      const int nbins = pass == 2 ? 1024 : 2048;
+      const uint32_t mask = (uint32_t)(nbins - 1);
+      for (int b = tid; b < nbins; b += kSmallThreads) s_hist[b] = 0u;
+      __syncthreads();
+      for (uint32_t base = 0; base < n; base += kSmallThreads * kLoads) {
+        uint2 e[kLoads];
+#pragma unroll
+        for (int u = 0; u < kLoads; ++u) {
+          const uint32_t i = base + u * kSmallThreads + tid;
+          e[u] = i < n ? c[i] : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kLoads; ++u) {
+          const bool in = base + u * kSmallThreads + tid < n;
+          if (in && (e[u].x & kAbsMask) == tau && (pass == 0 || (e[u].y >> prev_shift) == iprefix))
+            atomicAdd(&s_hist[(e[u].y >> shift) & mask], 1u);
+        }
+      }
+      __syncthreads();
+      uint32_t a = 0;
+      uint32_t idigit = pick_bin_1024(s_hist, nbins, false, t_rem, &a, s_warp, s_sel);
+      if (idigit == 0xFFFFFFFFu) { bad = true; idigit = 0u; a = 0u; }   // cannot happen: take <= n_equal
+      t_rem -= a;
+      iprefix = (iprefix << (pass == 2 ? 10 : 11)) | idigit;
+      __syncthreads();
+    }
+    idx_limit = iprefix;
+  }
+  // ---- votes
+  for (uint32_t base = 0; base < n; base += kSmallThreads * kLoads) {
+    uint2 e[kLoads];
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const uint32_t i = base + u * kSmallThreads + tid;
+      e[u] = i < n ? c[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < kLoads; ++u) {
+      const uint32_t key = e[u].x & kAbsMask;
+      if (base + u * kSmallThreads + tid < n && (key > tau || (key == tau && e[u].y <= idx_limit)))
+        add_vote(o.counter, o.packed, e[u].y, e[u].x >> 31);
+    }
+  }
+  if (tid == 0) {
+    rows[row].tau = tau;
+    rows[row].take_ties = take;
+    rows[row].n_emitted = bad ? 0xFFFFFFFFu : o.K;
+    if (bad) {
+      atomicAdd(hdr + kHdrBadCount, 1u);
+      atomicOr(hdr + kHdrStatus, (uint32_t)kFlagInternal);
+    }
+    atomicMax(hdr + kHdrMaxCand, rs.n_cand);
+  }
+}
+
 // kOrdered: the message (indices, sign bits) is wanted, so the candidates are laid out in index
 // order and emitted with their output positions.  Otherwise only the votes are wanted, whose
 // order does not matter: the candidates are copied as they lie, every entry above tau votes at
@@ -63,9 +216,21 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   __shared__ uint32_t s_sel[2];
   const uint32_t row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, lt = lanemask_lt();
   const RowState rs = rows[row];
-  if (kBin ? rs.done != kRowBin : (!row_uses_candidates(rs, o.K, cap) || !fits_single_cta(rs.n_cand))) return;
+  if (kBin ? rs.done != kRowBin : !row_uses_candidates(rs, o.K, cap)) return;
+  if (!kBin && !fits_single_cta(rs.n_cand)) {
+    // An unordered list (band form of the filter pass) cannot go through the general passes, which
+    // count and emit in index order: such a row is redone over the whole row.
+    if (o.unordered && tid == 0) rows[row].exact = 1u;
+    return;
+  }
   const uint32_t n = kBin ? (rs.n_bin < cap ? rs.n_bin : cap) : rs.n_cand;
-  const uint32_t k_want = kBin ? rs.k_rem : o.K;     // entries to keep out of the n
+  if (kBin && !fits_single_cta(n)) {                 // longer than this CTA's shared memory: select it where it lies
+    select_bin_in_place(rows, row, rs, cand + (uint64_t)row * cap, n, hdr, o, s_hist, s_warp, s_sel, rs.n_bin > cap);
+    return;
+  }
+  // entries to keep out of the n (whatever voted during the filter pass is no longer looked for; n_hi is 0
+  // unless that pass took its band form)
+  const uint32_t k_want = kBin ? rs.k_rem : o.K - rs.n_hi;
   uint32_t* s_bits = reinterpret_cast<uint32_t*>(smem_raw);   // [n] bit patterns, in ascending index order
   uint32_t* s_idx = s_bits + n;                               // [n] their indices
   const uint2* c = cand + (uint64_t)row * cap;
@@ -289,7 +454,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     if (tid == 0) {
       rows[row].tau = tau;
       rows[row].take_ties = take;
-      rows[row].n_emitted = kBin ? (n_kept == k_want ? o.K : n_kept) : n_kept;
+      rows[row].n_emitted = n_kept == k_want ? o.K : n_kept;
       if (!kBin) {                                               // a kRowBin row was counted when it was marked
         rows[row].done = 1u;
         atomicAdd(hdr + kHdrRowsDone, 1u);
@@ -385,7 +550,11 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
   const uint32_t n = rs.n_cand;
   const uint32_t per_cta = (n + C - 1) / C;
   // the same for every CTA of the cluster: either all go on or all leave
-  if (!row_uses_candidates(rs, o.K, cap) || (uint64_t)per_cta * 8u > (uint64_t)kSmallSelectBytes) return;
+  if (!row_uses_candidates(rs, o.K, cap)) return;
+  if ((uint64_t)per_cta * 8u > (uint64_t)kSmallSelectBytes) {
+    if (o.unordered && rank == 0 && tid == 0) rows[row].exact = 1u;   // see select_small_kernel
+    return;
+  }
   const uint32_t lo = rank * per_cta < n ? rank * per_cta : n;
   const uint32_t hi = lo + per_cta < n ? lo + per_cta : n;
   const uint32_t m = hi - lo;                                  // entries of this CTA
@@ -458,7 +627,7 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
   };
 
   // ---- tau = K-th largest magnitude of the row, take = how many entries equal to tau are kept
-  uint32_t prefix = 0, k_rem = o.K, n_equal = 0;
+  uint32_t prefix = 0, k_rem = o.K - rs.n_hi, n_equal = 0;
   for (int pass = 0; pass < kNumPasses; ++pass) {
     const int nbins = 1 << pass_bits(pass);
     const uint32_t mask = (uint32_t)(nbins - 1);
@@ -555,13 +724,15 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
   return e;
 }
 
-cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t* hdr, const EmitOut& o,
-                              cudaStream_t st) {
+cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin, uint32_t bin_cap, uint32_t* hdr,
+                              const EmitOut& o, cudaStream_t st) {
   auto kernel = select_small_kernel<false, true>;
   static int opted[kMaxDevices];
   cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)kSmallSelectBytes, opted);
   if (e != cudaSuccess) return e;
-  kernel<<<L.M, kSmallThreads, (size_t)L.bin_cap * 8u, st>>>(rows, bin, L.bin_cap, nullptr, 0u, hdr, o);
+  uint64_t need = (uint64_t)bin_cap * 8u;
+  if (need > kSmallSelectBytes) need = kSmallSelectBytes;
+  kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, bin, bin_cap, nullptr, 0u, hdr, o);
   e = cudaGetLastError();
   if (e == cudaSuccess) count_launch();
   return e;

@@ -81,6 +81,18 @@ def test_bad_arguments_rejected_before_launch(lib):
     assert lib.s3gd_step_randk(fake, fake, 1, 8, 2, 0.1, 1, 0, None, None, None, None, 1 << 30, None) == WS
 
 
+def test_exchange_calls_reject_bad_arguments(lib):
+    fake = ctypes.c_void_p(256 * 1024)
+    assert lib.s3gd_vote_apply(fake, fake, 0, 10, 1, 2, 8, 0.1, None, fake, 1 << 30, None) == 1       # no groups
+    assert lib.s3gd_vote_apply(fake, fake, 2, 1, 1, 2, 8, 0.1, None, fake, 1 << 30, None) == 1        # pieces overlap
+    assert lib.s3gd_vote_apply(fake, fake, 2, 10, 1, 2, 8, 0.1, None, fake, 8, None) == 2             # workspace too small
+    assert lib.s3gd_vote_counts(fake, fake, 200, 2, 8, 8, fake, 1, None, None) == 1                   # bytes cannot count 200 workers
+    assert lib.s3gd_vote_counts(fake, fake, 2, 2, 8, 6, fake, 4, None, None) == 1                     # padded length below d
+    assert lib.s3gd_vote_counts(fake, fake, 2, 2, 8, 8, fake, 2, None, None) == 1                     # counts are 1 or 4 bytes
+    assert lib.s3gd_encode_vote2(fake, 3, 1, 8, fake, None) == 1
+    assert lib.s3gd_apply_vote2(None, fake, 8, 0.1, None, None) == 1
+
+
 def test_binding_refuses_cpu_tensors(lib):
     import torch
     g = torch.zeros((2, 64))
