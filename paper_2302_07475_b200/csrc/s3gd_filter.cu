@@ -154,23 +154,29 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   }
   uint32_t result = 0xFFFFFFFFu;                   // no such bin: fewer than `want` samples in total
   if (searching && wsel != 0xFFFFFFFFu) {
-    // inside the chosen 1024 bins: 32 groups of 32 bins, from the top
-    for (int g = 31; g >= 0; --g) {
-      const uint32_t c = s_hist[wsel * 1024 + g * 32 + lane];
-      uint32_t suffix = c;                         // inclusive count of this bin and higher bins of the group
+    // inside the chosen 1024 bins: lane g sums group g (32 bins), a suffix scan over the lanes finds the
+    // group, a second one over that group's bins finds the bin -- two rounds instead of a walk over groups
+    const uint32_t* hb = s_hist + wsel * 1024;
+    uint32_t gsum = 0;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) gsum += hb[lane * 32 + ((i + lane) & 31)];      // staggered: no bank conflicts
+    uint32_t suffix = gsum;                          // entries in this group and the higher ones
 #pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
-        if (lane + s < 32) suffix += o;
-      }
-      const uint32_t gtot = __shfl_sync(0xFFFFFFFFu, suffix, 0);
-      if (above + gtot >= want) {
-        const uint32_t ok = __ballot_sync(0xFFFFFFFFu, above + suffix >= want);   // lanes 0..L satisfy it
-        result = wsel * 1024 + g * 32 + (31u - (uint32_t)__clz(ok));   // highest bin of the group that still reaches it
-        break;
-      }
-      above += gtot;
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
+      if (lane + s < 32) suffix += o;
     }
+    const uint32_t okg = __ballot_sync(0xFFFFFFFFu, above + suffix >= want);      // groups 0..G satisfy it (not empty)
+    const uint32_t g = 31u - (uint32_t)__clz(okg);
+    above += __shfl_sync(0xFFFFFFFFu, suffix - gsum, g);                          // entries in the groups above g
+    uint32_t bsuf = hb[g * 32 + lane];                                            // bins of group g, then their suffix sums
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, bsuf, s);
+      if (lane + s < 32) bsuf += o;
+    }
+    const uint32_t okb = __ballot_sync(0xFFFFFFFFu, above + bsuf >= want);        // bins 0..B of the group satisfy it
+    result = wsel * 1024 + g * 32 + (31u - (uint32_t)__clz(okb));
   }
   if (lane == 0 && warp == 0) s_res[0] = result == 0xFFFFFFFFu ? 0u : result << 16;   // too few samples: keep everything
   // bins run to 32767, so the bin above the highest one gives 0x80000000 = kNoPrevote by itself

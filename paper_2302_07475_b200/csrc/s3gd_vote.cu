@@ -126,9 +126,9 @@ __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_
                                                                    int8_t* __restrict__ opt_vote) {
   const uint64_t n_words = (d + 3) / 4;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-  const uint64_t gtid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  auto one_word = [&](uint64_t i, uint32_t w) {
-    if (w == kPackedZero && opt_vote == nullptr) return;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride) {
+    const uint32_t w = cw[i];
+    if (w == kPackedZero && opt_vote == nullptr) continue;
     int c[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) c[q] = (int)((w >> (8 * q)) & 0xFFu) - 128;
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_
         for (int q = 0; q < 4; ++q) pk |= (uint32_t)(uint8_t)(int8_t)((c[q] > 0) - (c[q] < 0)) << (8 * q);
         *reinterpret_cast<uint32_t*>(opt_vote + i * 4) = pk;
       }
-      if (w == kPackedZero) return;
+      if (w == kPackedZero) continue;
       float4* px = reinterpret_cast<float4*>(x + i * 4);
       float4 xv = *px;
       if (c[0]) xv.x = moved(xv.x, c[0], lr);
@@ -157,22 +157,7 @@ __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_
         if (c[q]) x[n] = moved(x[n], c[q], lr);
       }
     }
-  };
-  // four words (sixteen coordinates) per 16-byte load -- the counters start on a 16-byte boundary --
-  // and two such loads in flight; most words are untouched and cost nothing more
-  const uint64_t n_quads = n_words / 4;
-  const uint4* cw4 = reinterpret_cast<const uint4*>(cw);
-  for (uint64_t i4 = gtid; i4 < n_quads; i4 += 2 * stride) {
-    const uint4 a = cw4[i4];
-    const bool more = i4 + stride < n_quads;
-    const uint4 b = more ? cw4[i4 + stride] : make_uint4(kPackedZero, kPackedZero, kPackedZero, kPackedZero);
-    one_word(i4 * 4, a.x); one_word(i4 * 4 + 1, a.y); one_word(i4 * 4 + 2, a.z); one_word(i4 * 4 + 3, a.w);
-    if (more) {
-      const uint64_t j = (i4 + stride) * 4;
-      one_word(j, b.x); one_word(j + 1, b.y); one_word(j + 2, b.z); one_word(j + 3, b.w);
-    }
   }
-  if (gtid < n_words - n_quads * 4) one_word(n_quads * 4 + gtid, cw[n_quads * 4 + gtid]);
 }
 
 // err <- grads + eta * err: one rounding for the product, one for the sum (Eq. (5))
@@ -277,10 +262,8 @@ cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, 
   if (packed) {
     const uint32_t* cw = reinterpret_cast<const uint32_t*>(counter);
     const bool vecp = aligned(x, 16) && (opt_vote == nullptr || aligned(opt_vote, 4));
-    if (!aligned(cw, 16)) return cudaErrorMisalignedAddress;          // (the workspace region is 256-byte aligned)
-    const unsigned grid = grid_for(((d + 3) / 4 + 7) / 8, 256, sm_count() * 8);
-    if (vecp) counter_apply_packed_kernel<true><<<grid, 256, 0, st>>>(cw, x, d, lr, opt_vote);
-    else counter_apply_packed_kernel<false><<<grid, 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
     count_launch();
     return cudaGetLastError();
   }
