@@ -33,8 +33,8 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/, keyed by workload, with the digest of the kernel sources they were taken
 # at.  Reported only while the sources are unchanged.
 NCU_TRAFFIC = {
-    # 362.11 MB read+written for 8 rows (the ncu summary of the filter kernel under profiles/), traffic proportional to rows
-    "resnet18:11174": {"bytes": int(362.11e6 * 100 / 8), "digest": "35b76863fdbace2f"},
+    # 358.39 MB read + 4.49 MB written for 8 rows (profiles/filter_band_kernel_resnet18_M8.md), traffic proportional to rows
+    "resnet18:11174": {"bytes": int((358.391296e6 + 4.494080e6) * 100 / 8), "digest": "97245421bcc1d91c"},
 }
 KERNEL_SOURCES = ("s3gd_filter.cu", "s3gd_tile.cuh", "s3gd_common.cuh")
 
@@ -518,7 +518,9 @@ def run_ours(args):
                 models[k] += 8 * d
         mean_phase = [sum(p[k] for p in phases) / max(len(phases), 1) for k in range(5)]
         dominant = max(range(5), key=lambda k: mean_phase[k])
-        kernel_name = "signplane_step_kernel" if K == d else "filter_kernel"
+        kernel_name = "signplane_step_kernel" if K == d else "filter_band_kernel"
+        if args.unfused or args.error_feedback or sharded is not None:
+            kernel_name = "filter_kernel / filter_scan_kernel"      # the ranked form of the pass
         dom_ms = sum(kernel_ms) / max(len(kernel_ms), 1)      # from the timed steps
         b_grad = models["grad"]
         if args.randk:
