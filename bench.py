@@ -393,6 +393,9 @@ def run_ours(args):
     extended = args.error_feedback or args.momentum is not None
     err = torch.zeros((M, d), dtype=torch.float32, device=dev) if args.error_feedback else None
     vmom = torch.zeros(d, dtype=torch.float32, device=dev) if args.momentum is not None else None
+    # With error memory the same gradients every step would make every unkept coordinate grow in lockstep
+    # towards the threshold, which no training run does: alternate between two seeded batches instead.
+    grads_b = W.make_grads(spec, dev, step=1) if args.error_feedback else None
 
     step_no = [0]
     if args.unfused:                            # the three calls with the message written to device memory
@@ -417,7 +420,9 @@ def run_ours(args):
             step_no[0] += 1
             S.s3gd_step_randk(x, grads, K, spec.lr, 20230207, step_no[0], ws)
         elif extended:
-            S.s3gd_step_ex(x, grads, K, spec.lr, ws, err=err, eta=1.0, v=vmom, mu=args.momentum or 0.0)
+            step_no[0] += 1
+            g_now = grads_b if (grads_b is not None and step_no[0] % 2 == 0) else grads
+            S.s3gd_step_ex(x, g_now, K, spec.lr, ws, err=err, eta=1.0, v=vmom, mu=args.momentum or 0.0)
         else:
             S.s3gd_step(x, grads, K, spec.lr, ws)
 

@@ -68,12 +68,34 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   for (uint32_t b = tid; b < (uint32_t)kHistBins; b += 1024) hist[(uint64_t)row * kHistBins + b] = 0u;
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
   __syncthreads();
-  if (stride == 0) {                              // short row: every entry is inspected
-    for (uint32_t e = tid; e < n_sample; e += 1024) {
-      const uint32_t b = kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e];
-      atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u);
+  // every sampled entry of the row, in the scalar form (short rows, and the error-compensated step,
+  // whose row is formed on the fly from two buffers)
+  auto visit_samples = [&](auto&& visit) {
+    if (stride == 0) {                            // short row: every entry is inspected
+      for (uint32_t e = tid; e < n_sample; e += 1024) visit(kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e]);
+      return;
     }
-  } else if (!kEF) {
+    const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
+    for (uint32_t c0 = warp; c0 < n_chunks; c0 += 32 * kSampleUnroll) {
+      uint32_t v[kSampleUnroll];
+#pragma unroll
+      for (int u = 0; u < kSampleUnroll; ++u) {
+        const uint32_t c = c0 + 32 * u;
+        if (c < n_chunks) {
+          // offset inside the stride: hash scaled into [0, stride - 31) by a multiply-high (no division)
+          const uint64_t pos = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk - 1)) + lane;
+          v[u] = __ldg(rowp + pos);
+          if (kEF) v[u] = ef_value(v[u], __ldg(errp + pos), eta);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kSampleUnroll; ++u)
+        if (c0 + 32 * u < n_chunks) visit(v[u]);
+    }
+  };
+  if (stride == 0 || kEF) {
+    visit_samples([&](uint32_t b) { atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u); });
+  } else {
     // chunk c: 32 neighbours starting in [c*stride, (c+1)*stride - 32], on a 16-byte boundary so that a
     // lane reads four of them at once; eight lanes per chunk, four chunks per warp and load
     const uint32_t n_chunks = n_sample / kChunk;
@@ -102,24 +124,6 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
         }
       }
     }
-  } else {
-    const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
-    for (uint32_t c0 = warp; c0 < n_chunks; c0 += 32 * kSampleUnroll) {
-      uint32_t v[kSampleUnroll];
-#pragma unroll
-      for (int u = 0; u < kSampleUnroll; ++u) {
-        const uint32_t c = c0 + 32 * u;
-        if (c < n_chunks) {
-          // offset inside the stride: hash scaled into [0, stride - 31) by a multiply-high (no division)
-          const uint64_t pos = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk - 1)) + lane;
-          v[u] = __ldg(rowp + pos);
-          if (kEF) v[u] = ef_value(v[u], __ldg(errp + pos), eta);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < kSampleUnroll; ++u)
-        if (c0 + 32 * u < n_chunks) atomicAdd(&s_hist[(v[u] & kAbsMask) >> 16], 1u);
-    }
   }
   __syncthreads();
 
@@ -135,6 +139,7 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   // warp 0 with want = j_rank (tau_lo is that bin's lower edge), warp 1 with want = j_hi + 1 (the bin above
   // it is the lowest one with at most j_hi sampled entries at or above its lower edge: tau_hi).
   __shared__ uint32_t s_res[2];
+  __shared__ uint32_t s_fine[2];                  // the bin of tau_lo and the number of sampled entries above it
   const bool searching = warp == 0 || (warp == 1 && j_hi != 0u);
   const uint32_t want = warp == 0 ? j_rank : j_hi + 1u;
   uint32_t wsel = 0xFFFFFFFFu, above = 0;
@@ -176,12 +181,56 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
       if (lane + s < 32) bsuf += o;
     }
     const uint32_t okb = __ballot_sync(0xFFFFFFFFu, above + bsuf >= want);        // bins 0..B of the group satisfy it
-    result = wsel * 1024 + g * 32 + (31u - (uint32_t)__clz(okb));
+    const uint32_t bsel = 31u - (uint32_t)__clz(okb);
+    result = wsel * 1024 + g * 32 + bsel;
+    // sampled entries in bins above the chosen one (for the refinement below)
+    above += __shfl_sync(0xFFFFFFFFu, bsuf, bsel) - hb[g * 32 + bsel];
   }
-  if (lane == 0 && warp == 0) s_res[0] = result == 0xFFFFFFFFu ? 0u : result << 16;   // too few samples: keep everything
+  if (lane == 0 && warp == 0) {
+    s_res[0] = result == 0xFFFFFFFFu ? 0u : result << 16;   // too few samples: keep everything
+    s_fine[0] = result;
+    s_fine[1] = above;
+  }
   // bins run to 32767, so the bin above the highest one gives 0x80000000 = kNoPrevote by itself
   if (lane == 0 && warp == 1) s_res[1] = !searching ? kNoPrevote : (result == 0xFFFFFFFFu ? 0u : (result + 1u) << 16);
   __syncthreads();
+  if (kEF && s_fine[0] != 0xFFFFFFFFu) {
+    // With error memory the magnitudes of the entries that were not kept climb towards the threshold step
+    // after step, so a bin of the first histogram (2^-7 relative width) just below the K-th magnitude can
+    // hold many times K entries, and a threshold on a bin edge would let all of them through.  Place it
+    // inside the bin: a second look at the sample counts the bin's entries by their next 8 bits, and tau_lo
+    // becomes the lower edge of the sub-bin that holds rank j (2^-15 relative).
+    const uint32_t bin = s_fine[0], above_bin = s_fine[1];
+    for (uint32_t b = tid; b < 256u; b += 1024) s_hist[b] = 0u;          // (both searches are past the barrier)
+    __syncthreads();
+    visit_samples([&](uint32_t b) {
+      const uint32_t key = b & kAbsMask;
+      if ((key >> 16) == bin) atomicAdd(&s_hist[(key >> 8) & 0xFFu], 1u);
+    });
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t c[8], mine = 0;                                           // lane l owns sub-bins 8l .. 8l + 7
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = s_hist[lane * 8 + i]; mine += c[i]; }
+      uint32_t suffix = mine;
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suffix, s);
+        if (lane + s < 32) suffix += o;
+      }
+      const uint32_t ok = __ballot_sync(0xFFFFFFFFu, above_bin + suffix >= j_rank);   // not empty: the bin holds rank j
+      const uint32_t lsel = ok ? 31u - (uint32_t)__clz(ok) : 0u;
+      if (lane == lsel) {
+        uint32_t a = above_bin + suffix - mine, sub = 0;
+        for (int i = 7; i >= 0; --i) {
+          if (a + c[i] >= j_rank) { sub = (uint32_t)i; break; }
+          a += c[i];
+        }
+        s_res[0] = (bin << 16) | ((lane * 8u + sub) << 8);
+      }
+    }
+    __syncthreads();
+  }
   if (tid == 0) {
     rows[row].tau_lo = s_res[0];
     rows[row].tau_hi = s_res[1] > s_res[0] ? s_res[1] : s_res[0];      // never below tau_lo: what votes early has passed the filter

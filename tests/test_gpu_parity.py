@@ -478,6 +478,31 @@ def test_error_memory_and_momentum_over_steps(K, eta, mu):
                 assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"step {step}: message differs"
 
 
+def test_error_memory_in_its_steady_state_keeps_the_single_read_route():
+    """Many steps with error memory: the entries that are not kept climb towards the threshold step after
+    step, so the magnitudes just below the K-th become dense.  The sampled threshold must still sit close
+    enough to the K-th magnitude that every row is served from its survivors (none redone over the whole
+    row), and x and the error memory must equal the oracle's after every tenth step."""
+    s = W.spec("small_cnn", d=300_007, M=4)
+    d, M, K, steps = s.d, s.M, 300, 160
+    batches = [W.make_grads(s, DEV, step=0), W.make_grads(s, DEV, step=1)]
+    x = W.make_x(s, DEV)
+    err = torch.zeros((M, d), device=DEV)
+    x_o, e_o = x.cpu().numpy(), np.zeros((M, d), np.float32)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    redone = 0
+    for step in range(steps):
+        g = batches[step % 2]
+        S.s3gd_step_ex(x, g, K, s.lr, ws, err=err, eta=1.0)
+        code, info = S.s3gd_device_status(ws)
+        redone += info[1]
+        x_o, e_o, _, _, _ = O.error_feedback_step(x_o, g.cpu().numpy(), e_o, 1.0, K, s.lr, topk=O.topk_sign_threshold)
+        if step % 10 == 9:
+            assert np.array_equal(bits(err.cpu().numpy()), bits(e_o)), f"step {step}: error memory differs"
+            assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)), f"step {step}: x differs"
+    assert redone == 0, f"{redone} rows were redone over the whole row in {steps} steps"
+
+
 def test_error_memory_with_its_own_alignment():
     """The error memory starts 4 bytes off the gradients' alignment: the step must not assume they match."""
     s = W.spec("resnet18", d=150_001, M=4)
