@@ -267,6 +267,20 @@ S3GD_API s3gd_status s3gd_debug_step(float* x, const float* grads, int M, uint64
  *   out_words       dev  [ceil(n / 16)]
  *   s3gd_apply_vote2: x[n] <- fl32(x[n] - lr * vote[n]) from the words, one rounding, unmoved bits left
  *                   alone; opt_vote (dev or NULL, [d] int8) receives the decoded vote.
+ *
+ * s3gd_encode_vote_sparse / s3gd_apply_vote_sparse -- the same message in the sparse form the paper's
+ * count assumes (Section 2.2: only the union of the workers' supports is sent): the coordinates with a
+ * non-zero vote, ascending, and one sign bit each, in the layout of a worker's message.
+ *   src, src_kind, n_summed, n   as for s3gd_encode_vote2: the votes (or sums) of n consecutive coordinates
+ *   index_base      the coordinate of src[0] (a server that owns one range of the coordinates passes its start)
+ *   out_piece       dev  [1 + cap + ceil(cap / 32)] uint32: the number of non-zero votes, then up to cap
+ *                   indices (index_base + position, ascending), then their sign words (bit j belongs to
+ *                   index j, lowest bits first, 1 = negative, padding 0).  If there are more than cap
+ *                   non-zero votes the count says so and only the first cap are listed: the caller compares.
+ *   ws, ws_bytes    dev  scratch of s3gd_sparse_workspace_bytes(n) bytes, 4-byte aligned
+ *   s3gd_apply_vote_sparse: applies n_pieces such pieces, piece_stride uint32 words apart (an all-gather of
+ *                   equal pieces), to x; an index >= d is skipped and counted in opt_bad_count (dev or NULL).
+ *                   A piece whose count exceeds cap is applied as far as it is listed.
  */
 S3GD_API s3gd_status s3gd_vote_apply(float* x, const uint32_t* msg, int n_groups, uint64_t group_stride, int M_group,
                                      uint64_t K, uint64_t d, float lr, int8_t* opt_vote,
@@ -278,6 +292,13 @@ S3GD_API s3gd_status s3gd_encode_vote2(const void* src, int src_kind, uint32_t n
                                        uint32_t* out_words, void* stream);
 S3GD_API s3gd_status s3gd_apply_vote2(float* x, const uint32_t* words, uint64_t d, float lr, int8_t* opt_vote,
                                       void* stream);
+S3GD_API size_t s3gd_sparse_workspace_bytes(uint64_t n);
+S3GD_API s3gd_status s3gd_encode_vote_sparse(const void* src, int src_kind, uint32_t n_summed, uint64_t n,
+                                             uint32_t index_base, uint32_t cap, uint32_t* out_piece,
+                                             void* ws, size_t ws_bytes, void* stream);
+S3GD_API s3gd_status s3gd_apply_vote_sparse(float* x, const uint32_t* pieces, int n_pieces, uint64_t piece_stride,
+                                            uint32_t cap, uint64_t d, float lr, uint32_t* opt_bad_count,
+                                            void* stream);
 
 /*
  * Majority vote without any caller-provided scratch (the paper has no counterpart: this is

@@ -28,7 +28,7 @@ EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd
            "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
            "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter", "s3gd_last_device_status",
            "s3gd_debug_topk_sign", "s3gd_debug_step", "s3gd_vote_apply", "s3gd_vote_counts", "s3gd_encode_vote2",
-           "s3gd_apply_vote2")
+           "s3gd_apply_vote2", "s3gd_sparse_workspace_bytes", "s3gd_encode_vote_sparse", "s3gd_apply_vote_sparse")
 
 
 class S3gdError(RuntimeError):
@@ -100,6 +100,12 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_encode_vote2.argtypes = [vp, ctypes.c_int, u32, u64, u32p, vp]
     lib.s3gd_apply_vote2.restype = ctypes.c_int
     lib.s3gd_apply_vote2.argtypes = [vp, u32p, u64, ctypes.c_float, vp, vp]
+    lib.s3gd_sparse_workspace_bytes.restype = sz
+    lib.s3gd_sparse_workspace_bytes.argtypes = [u64]
+    lib.s3gd_encode_vote_sparse.restype = ctypes.c_int
+    lib.s3gd_encode_vote_sparse.argtypes = [vp, ctypes.c_int, u32, u64, u32, u32, u32p, vp, sz, vp]
+    lib.s3gd_apply_vote_sparse.restype = ctypes.c_int
+    lib.s3gd_apply_vote_sparse.argtypes = [vp, u32p, ctypes.c_int, u64, u32, u64, ctypes.c_float, vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -284,6 +290,44 @@ def s3gd_apply_vote2(x: torch.Tensor, words2: torch.Tensor, lr: float, opt_vote:
     with torch.cuda.device(x.device):
         code = load().s3gd_apply_vote2(*args, _stream(x))
     _check("s3gd_apply_vote2", code)
+
+
+def sparse_piece_words(cap: int) -> int:
+    """uint32 words of one sparse message: its count, cap indices, ceil(cap / 32) sign words."""
+    return 1 + int(cap) + words(cap)
+
+
+def s3gd_sparse_workspace_bytes(n: int) -> int:
+    return int(load().s3gd_sparse_workspace_bytes(int(n)))
+
+
+def s3gd_encode_vote_sparse(src: torch.Tensor, out_piece: torch.Tensor, cap: int, ws: torch.Tensor,
+                            index_base: int = 0, n_summed: int = 1) -> None:
+    """Sparse form (count, ascending indices, sign words) of the votes in src: int32 sums, summed biased bytes or int8."""
+    n = src.numel()
+    if src.dtype == torch.int32:
+        kind, p = 0, _ptr(src, torch.int32, name="src")
+    elif src.dtype == torch.uint8:
+        kind, p = 1, _ptr(src, torch.uint8, name="src")
+    else:
+        kind, p = 2, _ptr(src, torch.int8, name="src")
+    args = (p, kind, n_summed, n, index_base, cap, _ptr(out_piece, torch.int32, sparse_piece_words(cap), "out_piece"),
+            _ptr(ws, torch.uint8, name="ws"), ws.numel())
+    with torch.cuda.device(src.device):
+        code = load().s3gd_encode_vote_sparse(*args, _stream(src))
+    _check("s3gd_encode_vote_sparse", code)
+
+
+def s3gd_apply_vote_sparse(x: torch.Tensor, pieces: torch.Tensor, n_pieces: int, piece_stride: int, cap: int, lr: float,
+                           opt_bad_count: Optional[torch.Tensor] = None) -> None:
+    """x <- x - lr * vote from n_pieces sparse messages lying piece_stride words apart."""
+    d = x.numel()
+    need = (n_pieces - 1) * piece_stride + sparse_piece_words(cap)
+    args = (_ptr(x, torch.float32, name="x"), _ptr(pieces, torch.int32, need, "pieces"), n_pieces, piece_stride, cap, d,
+            ctypes.c_float(lr), _ptr(opt_bad_count, torch.int32, 1, "opt_bad_count"))
+    with torch.cuda.device(x.device):
+        code = load().s3gd_apply_vote_sparse(*args, _stream(x))
+    _check("s3gd_apply_vote_sparse", code)
 
 
 PHASES = ("sample", "filter", "threshold", "emit", "apply")

@@ -102,6 +102,138 @@ __global__ void __launch_bounds__(256) apply2_kernel(float* __restrict__ x, cons
   }
 }
 
+
+// ---- the sparse form of the server's message: the coordinates with a non-zero vote, ascending, and
+// their sign bits, in the layout of a worker's message.  Three launches: non-zero votes per block of
+// kSparseBlock coordinates; exclusive scan of the block counts (one CTA); ordered emission.
+constexpr int kSparseThreads = 256;
+constexpr int kSparsePer = 16;                                     // consecutive coordinates per thread
+constexpr int kSparseBlock = kSparseThreads * kSparsePer;          // coordinates per block
+
+template <int kKind>
+__device__ __forceinline__ int vote_of(const void* __restrict__ src, uint32_t bias, uint64_t i) {
+  int c;
+  if (kKind == 0) c = static_cast<const int32_t*>(src)[i];
+  else if (kKind == 1) c = (int)(int8_t)(uint8_t)(static_cast<const uint8_t*>(src)[i] - bias);
+  else c = static_cast<const int8_t*>(src)[i];
+  return (c > 0) - (c < 0);
+}
+
+// bit q of the results: coordinate first + q has a non-zero vote / a negative one
+template <int kKind>
+__device__ __forceinline__ void thread_votes(const void* __restrict__ src, uint32_t bias, uint64_t n, uint64_t first,
+                                             uint32_t* moved, uint32_t* negative) {
+  uint32_t mv = 0, ng = 0;
+#pragma unroll
+  for (int q = 0; q < kSparsePer; ++q) {
+    const uint64_t i = first + q;
+    if (i < n) {
+      const int v = vote_of<kKind>(src, bias, i);
+      mv |= (uint32_t)(v != 0) << q;
+      ng |= (uint32_t)(v < 0) << q;
+    }
+  }
+  *moved = mv; *negative = ng;
+}
+
+__device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_t* s_warp, uint32_t* total) {
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) {
+    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, s);
+    if (lane >= (uint32_t)s) inc += o;
+  }
+  __syncthreads();
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  uint32_t off = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kSparseThreads / 32; ++w) {
+    const uint32_t c = s_warp[w];
+    if ((uint32_t)w < warp) off += c;
+    tot += c;
+  }
+  *total = tot;
+  return off + inc - v;
+}
+
+template <int kKind>
+__global__ void __launch_bounds__(kSparseThreads) sparse_count_kernel(const void* __restrict__ src, uint32_t bias,
+                                                                      uint64_t n, uint32_t* __restrict__ blk) {
+  __shared__ uint32_t s_warp[kSparseThreads / 32];
+  uint32_t mv, ng;
+  thread_votes<kKind>(src, bias, n, (uint64_t)blockIdx.x * kSparseBlock + (uint64_t)threadIdx.x * kSparsePer, &mv, &ng);
+  uint32_t total;
+  block_exclusive_scan_256((uint32_t)__popc(mv), s_warp, &total);
+  if (threadIdx.x == 0) blk[blockIdx.x] = total;
+}
+
+// blk[b] <- number of non-zero votes in the blocks before b; *out_count <- their total.  One CTA.
+__global__ void __launch_bounds__(kSparseThreads) sparse_scan_kernel(uint32_t* __restrict__ blk, uint32_t n_blocks,
+                                                                     uint32_t* __restrict__ out_count) {
+  __shared__ uint32_t s_warp[kSparseThreads / 32];
+  uint32_t carry = 0;
+  for (uint32_t base = 0; base < n_blocks; base += kSparseThreads) {
+    const uint32_t b = base + threadIdx.x;
+    const uint32_t v = b < n_blocks ? blk[b] : 0u;
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan_256(v, s_warp, &total);
+    if (b < n_blocks) blk[b] = carry + ex;
+    carry += total;
+  }
+  if (threadIdx.x == 0) *out_count = carry;
+}
+
+template <int kKind>
+__global__ void __launch_bounds__(kSparseThreads) sparse_emit_kernel(const void* __restrict__ src, uint32_t bias,
+                                                                     uint64_t n, uint32_t index_base,
+                                                                     const uint32_t* __restrict__ blk, uint32_t cap,
+                                                                     uint32_t* __restrict__ out_idx,
+                                                                     uint32_t* __restrict__ out_signbits) {
+  __shared__ uint32_t s_warp[kSparseThreads / 32];
+  const uint64_t first = (uint64_t)blockIdx.x * kSparseBlock + (uint64_t)threadIdx.x * kSparsePer;
+  uint32_t mv, ng;
+  thread_votes<kKind>(src, bias, n, first, &mv, &ng);
+  uint32_t total;
+  uint32_t pos = blk[blockIdx.x] + block_exclusive_scan_256((uint32_t)__popc(mv), s_warp, &total);
+  // a thread's entries are consecutive in the output: at most two sign words are touched
+  uint32_t w0 = pos >> 5, bits0 = 0, bits1 = 0;
+  while (mv) {
+    const uint32_t q = (uint32_t)__ffs((int)mv) - 1u;
+    if (pos < cap) {
+      out_idx[pos] = index_base + (uint32_t)(first + q);
+      const uint32_t bit = (ng >> q & 1u) << (pos & 31u);
+      if ((pos >> 5) == w0) bits0 |= bit; else bits1 |= bit;
+    }
+    ++pos;
+    mv &= mv - 1u;
+  }
+  if (bits0) atomicOr(out_signbits + w0, bits0);
+  if (bits1) atomicOr(out_signbits + w0 + 1, bits1);
+}
+
+// x <- x - lr * vote from n_pieces sparse messages, piece_stride words apart: a piece is its count, then
+// cap indices, then ceil(cap / 32) sign words.  One thread per (piece, entry).
+__global__ void __launch_bounds__(256) sparse_apply_kernel(float* __restrict__ x, const uint32_t* __restrict__ msg,
+                                                           uint32_t n_pieces, uint64_t piece_stride, uint32_t cap,
+                                                           uint64_t d, float lr, uint32_t* __restrict__ bad_count) {
+  const uint64_t total = (uint64_t)n_pieces * cap;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  uint32_t bad = 0;
+  for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
+    const uint64_t p = e / cap, j = e - p * cap;
+    const uint32_t* piece = msg + p * piece_stride;
+    const uint32_t count = piece[0] < cap ? piece[0] : cap;
+    if (j >= count) continue;
+    const uint32_t n = piece[1 + j];
+    const uint32_t neg = (piece[1 + cap + (j >> 5)] >> (j & 31)) & 1u;
+    if (n < d) x[n] = neg ? __fadd_rn(x[n], lr) : __fsub_rn(x[n], lr);
+    else ++bad;
+  }
+  if (bad && bad_count) atomicAdd(bad_count, bad);
+}
+
 }  // namespace
 }  // namespace s3gd
 
@@ -190,6 +322,53 @@ s3gd_status s3gd_apply_vote2(float* x, const uint32_t* words, uint64_t d, float 
     return S3GD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   apply2_kernel<<<grid_for((d + 15) / 16, 256, sm_count() * 8), 256, 0, st>>>(x, words, d, lr, opt_vote);
+  if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+  count_launch();
+  return S3GD_OK;
+}
+
+size_t s3gd_sparse_workspace_bytes(uint64_t n) {
+  if (n == 0 || n >= (1ull << 32)) return 0;
+  return (size_t)((n + kSparseBlock - 1) / kSparseBlock) * sizeof(uint32_t);
+}
+
+s3gd_status s3gd_encode_vote_sparse(const void* src, int src_kind, uint32_t n_summed, uint64_t n, uint32_t index_base,
+                                    uint32_t cap, uint32_t* out_piece, void* ws, size_t ws_bytes, void* stream) {
+  if (src == nullptr || out_piece == nullptr || n == 0 || n >= (1ull << 32) || cap == 0 || !aligned(out_piece, 4) ||
+      src_kind < 0 || src_kind > 2 || (uint64_t)index_base + n > (1ull << 32))
+    return S3GD_ERR_INVALID_ARG;
+  if (src_kind == 0 && !aligned(src, 4)) return S3GD_ERR_INVALID_ARG;
+  const size_t need = s3gd_sparse_workspace_bytes(n);
+  if (ws == nullptr || ws_bytes < need || !aligned(ws, 4)) return S3GD_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* blk = static_cast<uint32_t*>(ws);
+  const uint32_t n_blocks = (uint32_t)((n + kSparseBlock - 1) / kSparseBlock);
+  const uint32_t bias = (128u * n_summed) & 0xFFu;
+  uint32_t* out_idx = out_piece + 1;
+  uint32_t* out_sgn = out_piece + 1 + cap;
+  if (cudaMemsetAsync(out_sgn, 0, (size_t)((cap + 31) / 32) * sizeof(uint32_t), st) != cudaSuccess) return S3GD_ERR_CUDA;
+  if (src_kind == 0) sparse_count_kernel<0><<<n_blocks, kSparseThreads, 0, st>>>(src, 0u, n, blk);
+  else if (src_kind == 1) sparse_count_kernel<1><<<n_blocks, kSparseThreads, 0, st>>>(src, bias, n, blk);
+  else sparse_count_kernel<2><<<n_blocks, kSparseThreads, 0, st>>>(src, 0u, n, blk);
+  sparse_scan_kernel<<<1, kSparseThreads, 0, st>>>(blk, n_blocks, out_piece);
+  if (src_kind == 0) sparse_emit_kernel<0><<<n_blocks, kSparseThreads, 0, st>>>(src, 0u, n, index_base, blk, cap, out_idx, out_sgn);
+  else if (src_kind == 1) sparse_emit_kernel<1><<<n_blocks, kSparseThreads, 0, st>>>(src, bias, n, index_base, blk, cap, out_idx, out_sgn);
+  else sparse_emit_kernel<2><<<n_blocks, kSparseThreads, 0, st>>>(src, 0u, n, index_base, blk, cap, out_idx, out_sgn);
+  if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
+  count_launch(3);
+  return S3GD_OK;
+}
+
+s3gd_status s3gd_apply_vote_sparse(float* x, const uint32_t* pieces, int n_pieces, uint64_t piece_stride, uint32_t cap,
+                                   uint64_t d, float lr, uint32_t* opt_bad_count, void* stream) {
+  if (x == nullptr || pieces == nullptr || n_pieces <= 0 || cap == 0 || d == 0 || d >= (1ull << 32) || !aligned(x, 4) ||
+      !aligned(pieces, 4) || piece_stride < 1ull + cap + (cap + 31) / 32)
+    return S3GD_ERR_INVALID_ARG;
+  if (opt_bad_count != nullptr && !aligned(opt_bad_count, 4)) return S3GD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (opt_bad_count && cudaMemsetAsync(opt_bad_count, 0, sizeof(uint32_t), st) != cudaSuccess) return S3GD_ERR_CUDA;
+  sparse_apply_kernel<<<grid_for((uint64_t)n_pieces * cap, 256, sm_count() * 16), 256, 0, st>>>(
+      x, pieces, (uint32_t)n_pieces, piece_stride, cap, d, lr, opt_bad_count);
   if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
   count_launch();
   return S3GD_OK;

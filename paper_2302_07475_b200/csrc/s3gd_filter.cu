@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
 }
 
 
-// ---- the band form of the pass, for the fused step without outputs where survivors are dense.
+// ---- the band form of the pass, for every fused step that wants only the votes (no message, no error memory).
 // Two thresholds come from the sample: tau_lo as above and tau_hi, placed so that (with the same
 // confidence) FEWER than K entries of the row lie at or above it.  Those entries are the largest
 // of the row, hence part of its top K whenever there are at most K of them, so they vote at once
@@ -543,14 +543,16 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
 // instructions per entry, because with survivors in nearly every 128-entry step the ranked forms
 // are bound by instruction issue, not by memory:
 //   A  a lane takes the largest magnitude of its four entries of a step (three max operations that
-//      keep NaN) and compares once; only a lane that has a survivor looks closer and pushes it
-//      (bit pattern, index) onto the CTA's queue with one shared-memory atomic;
+//      keep NaN) and compares once; the warp branches together if any lane has a survivor, and only
+//      then are the four entries tested one by one and the survivors pushed (bit pattern, index) onto
+//      the CTA's queue with one shared-memory atomic each;
 //   C  after the tile's one barrier all threads drain the queue side by side, one entry each: an
 //      entry at or above tau_hi votes, a band entry moves to the CTA's band buffer;
 //   D  one tile later the band buffer's count is final and thread 0 claims room in the row's list;
 //   F  another tile later the claim has returned and the buffer is copied out, coalesced.
 // Three buffers of each kind, so that a buffer is never refilled before its readers have passed
-// the next barrier.  Whatever does not fit a buffer is handled entry by entry at once (rare).
+// the next barrier.  A tile that pushes more than the queue holds is redone entry by entry after the
+// barrier; a band entry that finds the band buffer full claims its place in the row's list by itself (rare).
 
 __device__ __forceinline__ float max_keep_nan(float a, float b) {   // maximum that is NaN if either operand is
   float r;

@@ -1,7 +1,7 @@
 """Workers spread over several GPUs: the deployment shape of Algorithm 1.
 
 Every rank (one process per GPU) holds the gradients of its own ``M_local`` workers and a replica of x.
-Two ways through one step, chosen with ``downlink``:
+Three ways through one step, chosen with ``downlink``:
 
 ``"replicated"`` -- the uplink of Section 2.2 is the only exchange.
     1. TopKSign of the local rows into this rank's piece of the message: K uint32 indices and
@@ -25,6 +25,12 @@ Two ways through one step, chosen with ``downlink``:
     Bytes received per rank and step: about d (bytes) or 4d (int32) + d / 4, whatever M and K.
     Best once M K reaches a fraction of d.
 
+``"sparse"`` -- as ``"two_bit"`` up to the reduce-scatter; then every rank lists the non-zero votes of its range
+    (``s3gd_encode_vote_sparse``: count, ascending coordinates, one sign bit each -- the form Section 2.2's
+    downlink count assumes), the fixed-size pieces are all-gathered and applied (``s3gd_apply_vote_sparse``).
+    A piece has room for min(range length, world * M_local * K) votes, which is all a range can receive.
+    Smaller than the two-bit form when fewer than about one coordinate in 16 is voted on.
+
 This module is host-side ordering and buffer management; all arithmetic stays in the CUDA library.
 ``ops`` exists so that the rank logic (buffer layout, order of the gathered pieces, padding of the
 coordinate ranges) can be exercised on CPU ranks with other implementations of the calls; the
@@ -39,7 +45,7 @@ import torch.distributed as dist
 
 from . import binding
 
-DOWNLINKS = ("replicated", "two_bit")
+DOWNLINKS = ("replicated", "two_bit", "sparse")
 
 
 class ShardedStep:
@@ -87,12 +93,23 @@ class ShardedStep:
             cdtype = torch.uint8 if self.count_bytes else torch.int32
             self.counts = torch.empty(self.d_padded, dtype=cdtype, device=dev)
             self.counts_mine = torch.empty(self.range_len, dtype=cdtype, device=dev)
-            self.words2_mine = torch.empty(self.range_len // 16, dtype=torch.int32, device=dev)
-            self.words2_all = torch.empty(self.d_padded // 16, dtype=torch.int32, device=dev)
+            if downlink == "two_bit":
+                self.words2_mine = torch.empty(self.range_len // 16, dtype=torch.int32, device=dev)
+                self.words2_all = torch.empty(self.d_padded // 16, dtype=torch.int32, device=dev)
+            else:
+                self.sparse_cap = max(1, min(self.range_len, self.M * K))
+                self.piece2_words = binding.sparse_piece_words(self.sparse_cap)
+                self.sparse_mine = torch.empty(self.piece2_words, dtype=torch.int32, device=dev)
+                self.sparse_all = torch.empty(self.world * self.piece2_words, dtype=torch.int32, device=dev)
+                self.sparse_ws = torch.empty(max(self.ops.s3gd_sparse_workspace_bytes(self.range_len), 4),
+                                             dtype=torch.uint8, device=dev)
 
     def describe(self) -> str:
         if self.downlink == "replicated":
             return "s3gd_topk_sign + one all-gather of the message + s3gd_vote_apply"
+        if self.downlink == "sparse":
+            return ("s3gd_topk_sign + s3gd_vote_counts + reduce-scatter of the sums + s3gd_encode_vote_sparse + "
+                    "all-gather of the sparse vote + s3gd_apply_vote_sparse")
         return ("s3gd_topk_sign + s3gd_vote_counts + reduce-scatter of the sums + s3gd_encode_vote2 + "
                 "all-gather of the two-bit vote + s3gd_apply_vote2")
 
@@ -100,7 +117,8 @@ class ShardedStep:
         """Bytes each rank contributes to the exchange per step."""
         if self.downlink == "replicated":
             return 4 * self.piece_words
-        return self.d_padded * (1 if self.count_bytes else 4) + self.range_len // 4
+        down = self.range_len // 4 if self.downlink == "two_bit" else 4 * self.piece2_words
+        return self.d_padded * (1 if self.count_bytes else 4) + down
 
     # row r * M_local + m of the gathered message is worker m of rank r
     def gathered_indices(self) -> torch.Tensor:
@@ -136,6 +154,15 @@ class ShardedStep:
             return
         self.ops.s3gd_vote_counts(self.idx_local, self.sgn_local, self.M_local, self.K, self.d, self.counts)
         self._reduce_scatter_sum(self.counts_mine, self.counts)
+        if self.downlink == "sparse":
+            self.ops.s3gd_encode_vote_sparse(self.counts_mine, self.sparse_mine, self.sparse_cap, self.sparse_ws,
+                                             index_base=self.rank * self.range_len, n_summed=self.world)
+            if self.collective:
+                dist.all_gather_into_tensor(self.sparse_all, self.sparse_mine, group=self.group)
+            else:
+                self.sparse_all.copy_(self.sparse_mine)
+            self.ops.s3gd_apply_vote_sparse(x, self.sparse_all, self.world, self.piece2_words, self.sparse_cap, lr)
+            return
         self.ops.s3gd_encode_vote2(self.counts_mine, self.words2_mine, n_summed=self.world)
         if self.collective:
             dist.all_gather_into_tensor(self.words2_all, self.words2_mine, group=self.group)

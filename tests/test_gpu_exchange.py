@@ -2,7 +2,8 @@
 
 s3gd_vote_apply (vote over a message gathered from several senders, fused with the update),
 s3gd_vote_counts (vote sums that add up across GPUs), s3gd_encode_vote2 / s3gd_apply_vote2 (the
-server's message in two bits per coordinate).  Everything is integer work or one fp32 rounding:
+server's message in two bits per coordinate), s3gd_encode_vote_sparse / s3gd_apply_vote_sparse (the
+same message as a list of coordinates and sign bits).  Everything is integer work or one fp32 rounding:
 tolerance 0.  The exchange itself is emulated on one GPU by laying the senders' pieces side by side,
 which is exactly what an all-gather produces, and by adding the senders' sums as a reduce-scatter would.
 """
@@ -148,3 +149,71 @@ def test_two_bit_form_of_an_int8_vote(d):
     assert np.all((bits(got) == bits(want)) | (np.isnan(got) & np.isnan(want)))
     v = vote.cpu().numpy()
     assert np.array_equal(bits(got)[v == 0], xb[v == 0]) and np.array_equal(back.cpu().numpy(), v)
+
+
+def _sparse_piece(vote_np, cap, index_base=0):
+    """The oracle's sparse form laid out as the library's piece: count, cap indices, sign words."""
+    idx, sgn = O.encode_vote_sparse(vote_np)
+    piece = np.zeros(S.binding.sparse_piece_words(cap), np.uint32)
+    piece[0] = idx.shape[0]
+    n = min(idx.shape[0], cap)
+    piece[1:1 + n] = idx[:n] + np.uint32(index_base)
+    full = O.pack_sign_bits(vote_np[idx[:n].astype(np.int64)] < 0) if n else np.zeros(0, np.uint32)
+    piece[1 + cap:1 + cap + full.shape[0]] = full
+    return piece
+
+
+def _same_piece(got, want, cap):
+    """Count, the listed indices and every sign word must agree; index slots beyond the count are unspecified."""
+    n = min(int(want[0]), cap)
+    return got[0] == want[0] and np.array_equal(got[1:1 + n], want[1:1 + n]) and np.array_equal(got[1 + cap:], want[1 + cap:])
+
+
+@pytest.mark.parametrize("d,density,cap", [(1, 1.0, 4), (4095, 0.3, 4095), (4097, 0.02, 200), (100_003, 0.05, 6_000),
+                                           (100_003, 0.5, 1_000), (1_000_003, 0.001, 2_048)])
+def test_sparse_form_of_the_vote(d, density, cap):
+    gen = torch.Generator(DEV).manual_seed(d + cap)
+    moved = torch.rand(d, generator=gen, device=DEV) < density
+    sign = torch.where(torch.rand(d, generator=gen, device=DEV) < 0.5, -1, 1).to(torch.int8)
+    vote = torch.where(moved, sign, torch.zeros_like(sign))
+    v = vote.cpu().numpy()
+    ws = torch.empty(max(S.s3gd_sparse_workspace_bytes(d), 4), dtype=torch.uint8, device=DEV)
+    for src, n_summed in ((vote, 1), (vote.to(torch.int32) * 3, 1),
+                          (((vote.to(torch.int64) * 2 + 128 * 3) % 256).to(torch.uint8), 3)):     # int8 votes, int32 sums, summed bytes
+        piece = torch.full((S.binding.sparse_piece_words(cap),), -1, dtype=torch.int32, device=DEV)
+        S.s3gd_encode_vote_sparse(src, piece, cap, ws, index_base=0, n_summed=n_summed)
+        torch.cuda.synchronize()
+        assert _same_piece(u32(piece), _sparse_piece(v, cap), cap), f"source {src.dtype}"
+    # a range that does not start at coordinate 0, applied next to a second piece for the coordinates before it
+    half = d // 2
+    lo_piece = torch.from_numpy(_sparse_piece(v[:half], cap).view(np.int32).copy()).to(DEV) if half else None
+    hi_piece = torch.empty(S.binding.sparse_piece_words(cap), dtype=torch.int32, device=DEV)
+    S.s3gd_encode_vote_sparse(vote[half:].contiguous(), hi_piece, cap, ws, index_base=half)
+    torch.cuda.synchronize()
+    assert _same_piece(u32(hi_piece), _sparse_piece(v[half:], cap, index_base=half), cap)
+    if half and np.count_nonzero(v[:half]) <= cap and np.count_nonzero(v[half:]) <= cap:
+        stride = S.binding.sparse_piece_words(cap) + 3
+        both = torch.zeros(2 * stride, dtype=torch.int32, device=DEV)
+        both[:lo_piece.numel()] = lo_piece
+        both[stride:stride + hi_piece.numel()] = hi_piece
+        x = torch.linspace(-1, 1, d, device=DEV)
+        x_o = O.apply_vote(x.cpu().numpy(), v, 0.125)
+        bad = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+        S.s3gd_apply_vote_sparse(x, both, 2, stride, cap, 0.125, bad)
+        torch.cuda.synchronize()
+        assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)) and int(bad.item()) == 0
+
+
+def test_sparse_apply_skips_an_index_out_of_range():
+    d, cap = 50, 8
+    piece = np.zeros(S.binding.sparse_piece_words(cap), np.uint32)
+    piece[0] = 3
+    piece[1:4] = [2, 49, 50]
+    piece[1 + cap] = 0b010
+    x = torch.zeros(d, device=DEV)
+    bad = torch.zeros(1, dtype=torch.int32, device=DEV)
+    S.s3gd_apply_vote_sparse(x, torch.from_numpy(piece.view(np.int32).copy()).to(DEV), 1, piece.shape[0], cap, 0.5, bad)
+    torch.cuda.synchronize()
+    want = np.zeros(d, np.float32)
+    want[2], want[49] = -0.5, 0.5
+    assert np.array_equal(x.cpu().numpy(), want) and int(bad.item()) == 1

@@ -355,6 +355,26 @@ def test_forced_bad_threshold_takes_the_whole_row_route(name, d, M, K, sample_ra
     assert info[1] == 0 and np.array_equal(bits(xc.cpu().numpy()), bits(x_o))
 
 
+@pytest.mark.parametrize("name,d,M,K", [("large", 1_000_003, 3, 80_000), ("resnet50_ties", 2_000_005, 4, 150_000)])
+def test_votes_only_step_with_hardly_any_early_votes(name, d, M, K):
+    """K = 8 % of d and the early-vote threshold forced to the largest sampled magnitude: nearly every
+    survivor of the filter pass has to be listed (800 per 8192-entry tile, more than the per-tile band
+    buffer of the kernel holds but fewer than its queue), so the entries beyond the buffer take their places
+    in the list one by one.  Nothing may be redone and x must equal the oracle's."""
+    s = W.spec(name, d=d, M=M)
+    g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+    idx_o, sgn_o = O.topk_sign_threshold(g.cpu().numpy(), K)
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, M, K, d)
+    x_o = O.apply_vote(x.cpu().numpy(), vote_o, s.lr)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    for prevote_rank in (1, 0):                       # hardly any early votes, then the library's own threshold
+        xa = x.clone()
+        S.s3gd_debug_step(xa, g, K, s.lr, ws, 0, prevote_rank=prevote_rank)
+        code, info = S.s3gd_device_status(ws)
+        assert info[1] == 0, f"{info[1]} rows were redone (early-vote rank {prevote_rank})"
+        assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"x differs (early-vote rank {prevote_rank})"
+
+
 @pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900), (5_000, 2_500), (1025, 1)])
 def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
     """Many entries exactly at the K-th magnitude, more than are taken: the lowest indices must win.

@@ -91,6 +91,12 @@ def test_exchange_calls_reject_bad_arguments(lib):
     assert lib.s3gd_vote_counts(fake, fake, 2, 2, 8, 8, fake, 2, None, None) == 1                     # counts are 1 or 4 bytes
     assert lib.s3gd_encode_vote2(fake, 3, 1, 8, fake, None) == 1
     assert lib.s3gd_apply_vote2(None, fake, 8, 0.1, None, None) == 1
+    assert lib.s3gd_sparse_workspace_bytes(0) == 0 and lib.s3gd_sparse_workspace_bytes(4096) == 4
+    assert lib.s3gd_sparse_workspace_bytes(4097) == 8
+    assert lib.s3gd_encode_vote_sparse(fake, 2, 1, 8, 0, 0, fake, fake, 64, None) == 1               # no room at all
+    assert lib.s3gd_encode_vote_sparse(fake, 2, 1, 8, 0, 4, fake, fake, 2, None) == 2                # scratch too small
+    assert lib.s3gd_encode_vote_sparse(fake, 2, 1, 8, 0xFFFFFFFF, 4, fake, fake, 64, None) == 1      # coordinates past 2^32
+    assert lib.s3gd_apply_vote_sparse(fake, fake, 2, 5, 8, 100, 0.1, None, None) == 1                # pieces overlap
 
 
 def test_binding_refuses_cpu_tensors(lib):

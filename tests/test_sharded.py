@@ -75,6 +75,37 @@ class OracleOps:
         out_words.copy_(torch.from_numpy(O.encode_vote_2bit(vote).view(np.int32).copy()))
 
     @staticmethod
+    def s3gd_sparse_workspace_bytes(n):
+        return 4
+
+    @staticmethod
+    def s3gd_encode_vote_sparse(src, out_piece, cap, ws, index_base=0, n_summed=1):
+        from oracle import s3gd_oracle as O
+        a = src.numpy()
+        if src.dtype == torch.uint8:
+            a = ((a.astype(np.int64) - 128 * n_summed) % 256).astype(np.uint8).view(np.int8)
+        idx, sgn = O.encode_vote_sparse(np.sign(a.astype(np.int64)).astype(np.int8))
+        piece = np.zeros(out_piece.numel(), dtype=np.uint32)
+        piece[0] = idx.shape[0]
+        assert idx.shape[0] <= cap
+        piece[1:1 + idx.shape[0]] = idx + np.uint32(index_base)
+        piece[1 + cap:1 + cap + sgn.shape[0]] = sgn
+        out_piece.copy_(torch.from_numpy(piece.view(np.int32).copy()))
+
+    @staticmethod
+    def s3gd_apply_vote_sparse(x, pieces, n_pieces, piece_stride, cap, lr, opt_bad_count=None):
+        from oracle import s3gd_oracle as O
+        m = pieces.numpy().view(np.uint32)
+        vote = np.zeros(x.numel(), dtype=np.int8)
+        for p in range(n_pieces):
+            piece = m[p * piece_stride:(p + 1) * piece_stride]
+            n = int(piece[0])
+            part = O.decode_vote_sparse(piece[1:1 + n], piece[1 + cap:1 + cap + (n + 31) // 32], x.numel())
+            assert not np.any((vote != 0) & (part != 0))            # the ranges do not overlap
+            vote += part
+        x.copy_(torch.from_numpy(O.apply_vote(x.numpy(), vote, lr)))
+
+    @staticmethod
     def s3gd_apply_vote2(x, words2, lr, opt_vote=None):
         from oracle import s3gd_oracle as O
         v = O.decode_vote_2bit(words2.numpy().view(np.uint32), x.numel())
@@ -101,13 +132,15 @@ def _cpu_rank(rank, world, port, out_dir):
     for _ in range(3):
         x_ref, idx_ref, sgn_ref, _ = O.step(x_ref, grads.numpy(), K, lr)
     ok, ok_rows = True, True
-    for downlink in ("replicated", "two_bit"):
+    for downlink in ("replicated", "two_bit", "sparse"):
         st = ShardedStep(M_local, d, K, "cpu", ops=OracleOps, downlink=downlink)
         assert st.M == world * M_local
         if downlink == "replicated":
             assert st.message_bytes_per_rank() == 4 * M_local * (K + 2)
-        else:                                       # d = 1003 over 2 ranks: ranges of 512 coordinates (a multiple of 16)
+        elif downlink == "two_bit":                 # d = 1003 over 2 ranks: ranges of 512 coordinates (a multiple of 16)
             assert st.range_len == 512 and st.d_padded == 1024 and st.message_bytes_per_rank() == 1024 + 128
+        else:                                       # room for min(512, 6 workers x 37) = 222 votes per range
+            assert st.sparse_cap == 222 and st.message_bytes_per_rank() == 1024 + 4 * (1 + 222 + 7)
         x_rank = x.clone()
         for _ in range(3):
             st.step(x_rank, mine, lr)
@@ -134,7 +167,7 @@ def test_two_cpu_ranks_match_the_single_process_step(tmp_path):
         assert open(tmp_path / f"r{r}.txt").read() == "1 1 1"
 
 
-@pytest.mark.parametrize("downlink", ["replicated", "two_bit"])
+@pytest.mark.parametrize("downlink", ["replicated", "two_bit", "sparse"])
 def test_without_a_process_group_it_is_the_plain_step(downlink):
     from oracle import s3gd_oracle as O
     from paper_2302_07475_b200.sharded import ShardedStep
@@ -189,7 +222,7 @@ def _gpu_rank(rank, world, port, out_dir):
     grads, x = W.make_grads(s, dev), W.make_x(s, dev)
     K = 3000
     ok = True
-    for downlink in ("replicated", "two_bit"):
+    for downlink in ("replicated", "two_bit", "sparse"):
         st = ShardedStep(s.M, s.d, K, dev, downlink=downlink)
         xr = x.clone()
         x_ref = x.cpu().numpy()
