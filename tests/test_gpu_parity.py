@@ -375,6 +375,55 @@ def test_votes_only_step_with_hardly_any_early_votes(name, d, M, K):
         assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"x differs (early-vote rank {prevote_rank})"
 
 
+@pytest.mark.parametrize("seed", range(60))
+def test_random_shapes_data_and_forced_ranks(seed):
+    """A sweep over what the other tests fix by hand: random row lengths beyond the sample size, worker
+    counts, K from 1 to d/4, four kinds of data (Gaussian, heavy-tailed with block scales, a handful of
+    magnitude levels so that ties abound, long constant stretches) and random sampling ranks for both
+    thresholds, so that good guesses, every kind of bad guess and their mixtures within one batch all occur.
+    Whatever route each row takes, the message, the votes and x must equal the oracle's."""
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.integers(131_073, 420_000))
+    M = int(rng.integers(1, 7))
+    K = int(rng.choice([1, 17, d // 1000, d // 100, d // 20, d // 4]))
+    kind = seed % 4
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    if kind == 1:
+        g = (rng.standard_t(2.5, (M, d)) * np.repeat(10.0 ** rng.uniform(-3, 0, 16), (d + 15) // 16)[:d]).astype(np.float32)
+    elif kind == 2:
+        g = (rng.choice(np.array([0.0, 0.25, 0.5, 1.0, 1.5, 3.0], np.float32), (M, d)) *
+             rng.choice(np.array([-1.0, 1.0], np.float32), (M, d))).astype(np.float32)
+    elif kind == 3:
+        g[:, d // 3: d // 3 + d // 5] = 2.5                       # a stretch of equal, large entries
+        g[M - 1, : d // 7] = -0.0
+    sample_rank = int(rng.choice([0, 0, 1, 40, 3_000, 65_536]))
+    prevote_rank = int(rng.choice([0, 0, 1, 9, 700, 30_000]))
+    gt = torch.from_numpy(g).to(DEV)
+    xt = torch.from_numpy(rng.standard_normal(d).astype(np.float32)).to(DEV)
+    idx_o, sgn_o = O.topk_sign_threshold(g, K)
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, M, K, d)
+    x_o = O.apply_vote(xt.cpu().numpy(), vote_o, 0.0625)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    ws.fill_(0xE1)
+    idx = torch.full((M, K), -1, dtype=torch.int32, device=DEV)
+    sgn = torch.full((M, S.binding.words(K)), -1, dtype=torch.int32, device=DEV)
+    vote = torch.full((d,), 77, dtype=torch.int8, device=DEV)
+    tag = f"d={d} M={M} K={K} kind={kind} ranks=({sample_rank}, {prevote_rank})"
+    S.s3gd_debug_topk_sign(gt, K, idx, sgn, ws, sample_rank)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"{tag}: message differs"
+    xa = xt.clone()
+    S.s3gd_debug_step(xa, gt, K, 0.0625, ws, sample_rank, prevote_rank=prevote_rank)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"{tag}: votes-only step differs"
+    idx.fill_(-1); sgn.fill_(-1)
+    xb = xt.clone()
+    S.s3gd_debug_step(xb, gt, K, 0.0625, ws, sample_rank, idx, sgn, vote, prevote_rank=prevote_rank)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o) and np.array_equal(vote.cpu().numpy(), vote_o), tag
+    assert np.array_equal(bits(xb.cpu().numpy()), bits(x_o)), f"{tag}: step with outputs differs"
+
+
 @pytest.mark.parametrize("n_ties,take", [(600, 300), (3000, 1500), (3000, 2999), (900, 900), (5_000, 2_500), (1025, 1)])
 def test_ties_at_the_threshold_in_a_row_that_fits_on_chip(n_ties, take):
     """Many entries exactly at the K-th magnitude, more than are taken: the lowest indices must win.
