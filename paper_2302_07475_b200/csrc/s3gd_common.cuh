@@ -124,9 +124,11 @@ constexpr uint32_t kRowTwoPass = 2u, kRowBin = 3u;
 // Does this row take its top-K from the filtered candidates (true) or from the whole row?
 // Band form: the n_hi entries at or above tau_hi have voted already.  They are the n_hi largest of
 // the row, so they belong to the top K exactly if n_hi <= K, and the other K - n_hi are then the
-// largest of the band, provided it holds that many.  (n_hi is 0 in the plain form.)
+// largest of the band, provided it holds that many.  (n_hi is 0 in the plain form.)  A row whose early
+// votes are exactly K has nothing left to select; the selections all look for at least one entry, so
+// that rare row is redone as well.
 __device__ __forceinline__ bool row_uses_candidates(const RowState& rs, uint32_t K, uint32_t cap) {
-  return rs.exact == 0u && rs.n_hi <= K && rs.n_cand >= K - rs.n_hi && rs.n_cand <= cap;
+  return rs.exact == 0u && rs.n_hi < K && rs.n_cand >= K - rs.n_hi && rs.n_cand <= cap;
 }
 // Shared memory the single-CTA selection needs for a row: bit pattern and index of every
 // candidate.  Rows that fit are finished by that kernel; the others by the general passes.

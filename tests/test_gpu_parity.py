@@ -375,6 +375,31 @@ def test_votes_only_step_with_hardly_any_early_votes(name, d, M, K):
         assert np.array_equal(bits(xa.cpu().numpy()), bits(x_o)), f"x differs (early-vote rank {prevote_rank})"
 
 
+def test_early_votes_that_are_exactly_the_top_k():
+    """Three tiers per row: K entries of magnitude 1000, as many of magnitude 10, the rest below 0.9.  With the
+    early-vote threshold forced between the two upper tiers, exactly K entries vote during the filter pass and
+    nothing is left to select: the row must end up with the oracle's x all the same (it is redone)."""
+    M, d, K = 3, 300_007, 2_000
+    gen = torch.Generator("cpu").manual_seed(77)
+    rows = []
+    for m in range(M):
+        v = 0.9 * torch.rand(d, generator=gen)
+        perm = torch.randperm(d, generator=gen)
+        v[perm[:K]] = 1000.0
+        v[perm[K:2 * K]] = 10.0
+        rows.append(v * torch.where(torch.rand(d, generator=gen) < 0.5, -1.0, 1.0))
+    g = torch.stack(rows).float().contiguous().to(DEV)
+    x = torch.zeros(d, device=DEV)
+    x_o, _, _, _ = O.step(x.cpu().numpy(), g.cpu().numpy(), K, 0.5)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    # about 437 of the 65,536 sampled entries per row are of the first tier and as many of the second: rank 650
+    # falls into the second tier, so the threshold sits on the upper edge of its histogram bin
+    S.s3gd_debug_step(x, g, K, 0.5, ws, 0, prevote_rank=650)
+    code, info = S.s3gd_device_status(ws)
+    assert code == 0 and info[1] == M
+    assert np.array_equal(bits(x.cpu().numpy()), bits(x_o))
+
+
 @pytest.mark.parametrize("seed", range(60))
 def test_random_shapes_data_and_forced_ranks(seed):
     """A sweep over what the other tests fix by hand: random row lengths beyond the sample size, worker
