@@ -624,6 +624,24 @@ def test_step_ex_without_options_is_the_plain_step():
     assert torch.equal(xa, xb)
 
 
+@pytest.mark.parametrize("K", [300, 9_000, 300_007])
+def test_momentum_without_error_memory_over_steps(K):
+    """The momentum update on top of the plain fused step (no error memory): x and v over carried steps."""
+    s = W.spec("resnet18", d=300_007, M=5)
+    d, M = s.d, s.M
+    x, v = W.make_x(s, DEV), torch.zeros(s.d, device=DEV)
+    x_o, v_o = x.cpu().numpy(), np.zeros(d, np.float32)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    for step in range(3):
+        g = W.make_grads(s, DEV, step=step)
+        S.s3gd_step_ex(x, g, K, s.lr, ws, v=v, mu=0.9)
+        S.s3gd_device_status(ws)
+        _, _, _, vote_o = O.step(x_o, g.cpu().numpy(), K, s.lr)
+        x_o, v_o = O.apply_vote_momentum(x_o, v_o, vote_o, 0.9, s.lr)
+        assert np.array_equal(bits(v.cpu().numpy()), bits(v_o)), f"step {step}: momentum differs"
+        assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)), f"step {step}: x differs"
+
+
 def test_unfused_momentum_update():
     d = 100_003
     gen = torch.Generator(DEV).manual_seed(5)
