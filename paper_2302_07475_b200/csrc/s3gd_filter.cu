@@ -614,9 +614,12 @@ __device__ __noinline__ uint32_t band_tile_slow(const uint32_t* __restrict__ row
 }
 
 // kThreads threads take tiles of 32 * kThreads entries (a warp owns 1024 contiguous ones, as in the
-// other forms).  Smaller CTAs, more of them per SM: fewer warps wait on each other at the tile's barrier.
+// other forms).  Measured on the resnet50 shape at K = 1 % (filter pass alone): 256 threads with 4 / 5 / 6
+// CTAs per SM 0.578 / 0.551 / 0.675 ms (56 / 46 / 40 registers); 128 and 64 threads with 8 and 16 CTAs per SM
+// 0.68 and 1.06 ms.  Five CTAs of 256 threads it is: 1280 threads per SM.
+constexpr int kBandThreadsPerSm = 1280;
 template <int kThreads>
-__global__ void __launch_bounds__(kThreads, 1024 / kThreads) filter_band_kernel(const uint32_t* __restrict__ gbits, int M,
+__global__ void __launch_bounds__(kThreads, kBandThreadsPerSm / kThreads) filter_band_kernel(const uint32_t* __restrict__ gbits, int M,
                                                                                 uint64_t d, RowState* __restrict__ rows,
                                                                                 uint2* __restrict__ cand, uint32_t cap,
                                                                                 int32_t* __restrict__ counter,
@@ -785,7 +788,7 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
   if (band) {                                    // (the caller asks for it only without error memory and with counters)
     constexpr int kBandThreads = 256;
     const uint64_t tiles = (uint64_t)L.M * ((L.d + kBandThreads * 32 - 1) / (kBandThreads * 32));
-    const uint64_t resident = (uint64_t)sm_count() * (1024 / kBandThreads);
+    const uint64_t resident = (uint64_t)sm_count() * (kBandThreadsPerSm / kBandThreads);
     filter_band_kernel<kBandThreads><<<(unsigned)(tiles < resident ? tiles : resident), kBandThreads, 0, st>>>(
         gbits, L.M, L.d, rows, cand, L.cap, zero_counter, packed ? 1u : 0u);
     return cudaGetLastError();
