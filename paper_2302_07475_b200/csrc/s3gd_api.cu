@@ -275,7 +275,7 @@ s3gd_status step_impl(float* x, const float* sel, float* err_to_clear, float* v,
   if (opt_signbits) S3GD_TRY(cudaMemsetAsync(opt_signbits, 0, (size_t)M * ((K + 31) / 32) * sizeof(uint32_t), st));
   S3GD_TRY(launch_select(sel, L, ws, opt_idx, opt_signbits, counter, packed, err_to_clear, ef_raw, eta, st));
   cudaError_t e = v ? launch_counter_apply_momentum(counter, packed, x, v, d, mu, lr, opt_vote, st)
-                    : launch_counter_apply(counter, packed, x, d, lr, opt_vote, st);
+                    : launch_counter_apply(counter, packed, x, d, lr, opt_vote, (uint64_t)M * K, st);
   prof_mark(kPhaseApplied, st);
   return from_cuda(e);
 }
@@ -386,7 +386,7 @@ s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uin
   for (int ph = kPhaseSampled; ph <= kPhaseThreshold; ++ph) prof_mark(ph, st);
   S3GD_TRY(launch_randk(grads, M, d, K, seed, step, opt_idx, opt_signbits, counter, packed, hdr, st));
   prof_mark(kPhaseEmitted, st);
-  cudaError_t e = launch_counter_apply(counter, packed, x, d, lr, opt_vote, st);
+  cudaError_t e = launch_counter_apply(counter, packed, x, d, lr, opt_vote, (uint64_t)M * K, st);
   prof_mark(kPhaseApplied, st);
   return from_cuda(e);
 }

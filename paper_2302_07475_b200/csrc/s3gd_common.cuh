@@ -170,8 +170,11 @@ cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cud
 cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,
                                 int32_t* counter, uint32_t* hdr, cudaStream_t st);
 cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st);
+// max_votes: an upper bound on the votes the counters hold (0 = unknown); when they are at most one per
+// kSparseVotesRatio coordinates the packed form is read in a way that suits mostly untouched counters
+constexpr uint64_t kSparseVotesRatio = 64;
 cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, uint64_t d, float lr, int8_t* opt_vote,
-                                 cudaStream_t st);
+                                 uint64_t max_votes, cudaStream_t st);
 cudaError_t launch_signplane_step(float* x, const float* grads, int M, uint64_t d, float lr, int8_t* opt_vote,
                                   cudaStream_t st);
 cudaError_t launch_signplane_message(const float* grads, int M, uint64_t d, uint32_t* out_idx,

@@ -269,7 +269,7 @@ s3gd_status s3gd_vote_apply(float* x, const uint32_t* msg, int n_groups, uint64_
     if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
     count_launch();
   }
-  return launch_counter_apply(counter, packed, x, d, lr, opt_vote, st) == cudaSuccess ? S3GD_OK : S3GD_ERR_CUDA;
+  return launch_counter_apply(counter, packed, x, d, lr, opt_vote, total, st) == cudaSuccess ? S3GD_OK : S3GD_ERR_CUDA;
 }
 
 s3gd_status s3gd_vote_counts(const uint32_t* idx, const uint32_t* signbits, int M, uint64_t K, uint64_t d,

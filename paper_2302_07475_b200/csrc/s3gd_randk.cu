@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(256) randk_kernel(const uint32_t* __restrict__
                                                     uint32_t* __restrict__ out_idx, uint32_t* __restrict__ out_signbits,
                                                     int32_t* __restrict__ counter, uint32_t packed,
                                                     uint32_t* __restrict__ hdr) {
-  const uint32_t words = (K + 31u) / 32u;
+  const uint32_t words = (uint32_t)(((uint64_t)K + 31u) / 32u);      // (K + 31 would wrap for K near 2^32)
   const uint64_t total = (uint64_t)words * (uint64_t)M;
   const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
   const uint32_t lane = lane_id();
@@ -65,10 +65,10 @@ __global__ void __launch_bounds__(256) randk_kernel(const uint32_t* __restrict__
     uint32_t key[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) key[r] = mix32(base + (uint32_t)(r + 1) * 0x9E3779B9u);
-    const uint32_t j = ww * 32u + lane;
+    const uint64_t j = (uint64_t)ww * 32u + lane;
     bool neg = false;
     if (j < K) {
-      const uint32_t n = permute(j, d, h, key, &gave_up);
+      const uint32_t n = permute((uint32_t)j, d, h, key, &gave_up);
       neg = (__ldg(gbits + (uint64_t)m * d + n) >> 31) != 0u;
       if (out_idx) out_idx[(uint64_t)m * K + j] = n;
       if (counter) add_vote(counter, packed, n, neg ? 1u : 0u);

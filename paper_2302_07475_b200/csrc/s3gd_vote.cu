@@ -160,6 +160,53 @@ __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_
   }
 }
 
+// Packed counters where few coordinates were voted on (at most one in 64): nearly every word is the
+// zero pattern, so the pass is a scan of d bytes whose speed is set by the bytes each thread keeps in
+// flight.  A thread loads two 16-byte groups (32 coordinates) at a time and only looks inside a group
+// that differs from the zero pattern.  x 16-byte aligned, no vote output.
+__global__ void __launch_bounds__(256) counter_apply_packed_sparse_kernel(const uint32_t* __restrict__ cw,
+                                                                          float* __restrict__ x, uint64_t d, float lr) {
+  const uint64_t n_words = (d + 3) / 4, n_groups = n_words / 4;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const uint64_t first = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const uint4* cg = reinterpret_cast<const uint4*>(cw);
+  auto word = [&](uint64_t i, uint32_t w) {       // word i = coordinates 4i .. 4i+3
+    if (w == kPackedZero) return;
+    int c[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) c[q] = (int)((w >> (8 * q)) & 0xFFu) - 128;
+    if (i * 4 + 4 <= d) {
+      float4* px = reinterpret_cast<float4*>(x + i * 4);
+      float4 xv = *px;
+      if (c[0]) xv.x = moved(xv.x, c[0], lr);
+      if (c[1]) xv.y = moved(xv.y, c[1], lr);
+      if (c[2]) xv.z = moved(xv.z, c[2], lr);
+      if (c[3]) xv.w = moved(xv.w, c[3], lr);
+      *px = xv;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t n = i * 4 + q;
+        if (n < d && c[q]) x[n] = moved(x[n], c[q], lr);
+      }
+    }
+  };
+  auto group = [&](uint64_t g, const uint4& v) {
+    if (v.x == kPackedZero && v.y == kPackedZero && v.z == kPackedZero && v.w == kPackedZero) return;
+    word(g * 4, v.x); word(g * 4 + 1, v.y); word(g * 4 + 2, v.z); word(g * 4 + 3, v.w);
+  };
+  uint64_t g = first;
+  for (; g + stride < n_groups; g += 2 * stride) {
+    const uint4 a = __ldcs(cg + g), b = __ldcs(cg + g + stride);
+    group(g, a);
+    group(g + stride, b);
+  }
+  if (g < n_groups) group(g, __ldcs(cg + g));
+  // the words after the last whole group
+  const uint64_t i = n_groups * 4 + first;
+  if (i < n_words) word(i, cw[i]);
+}
+
 // err <- grads + eta * err: one rounding for the product, one for the sum (Eq. (5))
 __global__ void __launch_bounds__(256) ef_accumulate_kernel(float* __restrict__ err, const float* __restrict__ grads,
                                                             float eta, uint64_t n) {
@@ -258,9 +305,15 @@ cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote
 }
 
 cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, uint64_t d, float lr, int8_t* opt_vote,
-                                 cudaStream_t st) {
+                                 uint64_t max_votes, cudaStream_t st) {
   if (packed) {
     const uint32_t* cw = reinterpret_cast<const uint32_t*>(counter);
+    if (max_votes != 0 && max_votes <= d / kSparseVotesRatio && opt_vote == nullptr && aligned(x, 16) &&
+        aligned(counter, 16)) {
+      counter_apply_packed_sparse_kernel<<<grid_for((d + 15) / 16, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr);
+      count_launch();
+      return cudaGetLastError();
+    }
     const bool vecp = aligned(x, 16) && (opt_vote == nullptr || aligned(opt_vote, 4));
     if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
     else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);

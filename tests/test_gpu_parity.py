@@ -179,11 +179,8 @@ def test_resnet50_tie_stress_full_size():
     _full_size("resnet50_ties", W.SPECS["resnet50_ties"].Ks, sample_rows=(31,))
 
 
-def _room_for_large_case():
-    """The d = 2.1e9, M = 8 case holds 67.2 GB of gradients, x twice, 8.7 GB of workspace and the message on
-    the device, and one 8.4 GB row plus the oracle's temporaries (about five times that) on the host."""
+def _room_for(need_dev, need_host):
     free_dev, _ = torch.cuda.mem_get_info()
-    need_dev = 100e9
     if free_dev < need_dev:
         return f"device has {free_dev / 1e9:.0f} GB free, the case needs {need_dev / 1e9:.0f} GB"
     try:
@@ -191,10 +188,15 @@ def _room_for_large_case():
         free_host = psutil.virtual_memory().available
     except Exception:
         return ""
-    need_host = 60e9
     if free_host < need_host:
         return f"host has {free_host / 1e9:.0f} GB available, the oracle needs {need_host / 1e9:.0f} GB for one row"
     return ""
+
+
+def _room_for_large_case():
+    """The d = 2.1e9, M = 8 case holds 67.2 GB of gradients, x twice, 8.7 GB of workspace and the message on
+    the device, and one 8.4 GB row plus the oracle's temporaries (about five times that) on the host."""
+    return _room_for(100e9, 60e9)
 
 
 def test_large_full_size_row_by_row():
@@ -233,6 +235,80 @@ def test_large_full_size_row_by_row():
     code, info = S.s3gd_device_status(ws)
     assert info[1] == 0
     assert np.array_equal(bits(x2.cpu().numpy()), bits(x_o))
+
+
+def test_longest_row_the_interface_accepts():
+    """d = 2^32 - 1, one worker: every index up to 4,294,967,294 must survive the 32-bit arithmetic of the kernels.
+    Large entries are planted at the very end of the row, around 2^31 and at the start, so the highest indices are
+    in the message.  The message is certified against the row by the oracle's O(d) certificate; with one worker the
+    vote is the worker's own TopKSign (Section 3.3, M = 1), which the oracle's vote and update turn into x."""
+    if os.environ.get("S3GD_TEST_LARGE") == "0":
+        pytest.skip("switched off with S3GD_TEST_LARGE=0")
+    why = _room_for(80e9, 75e9)
+    if why:
+        print("longest-row case skipped:", why)
+        pytest.skip(why)
+    d = (1 << 32) - 1
+    s = W.spec("large", d=d, M=1)
+    K = 4_294_967
+    g = W.make_grads(s, DEV)
+    planted = [0, 1, 31, (1 << 31) - 1, 1 << 31, (1 << 31) + 1, d - 8193, d - 8192, d - 130, d - 5, d - 4, d - 3, d - 2, d - 1]
+    g[0, torch.tensor(planted, device=DEV)] = torch.tensor([(-1.0) ** i * (100.0 + i) for i in range(len(planted))], device=DEV)
+    x = W.make_x(s, DEV)
+    x0 = x.clone()
+    lr = 0.5
+    ws = S.alloc_workspace(1, d, K, DEV)
+    idx = torch.empty((1, K), dtype=torch.int32, device=DEV)
+    sgn = torch.empty((1, S.binding.words(K)), dtype=torch.int32, device=DEV)
+    S.s3gd_step(x, g, K, lr, ws, idx, sgn, None)
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0
+    idx_g, sgn_g = u32(idx)[0].copy(), u32(sgn)[0].copy()
+    assert set(planted) <= set(idx_g[np.searchsorted(idx_g, planted).clip(max=K - 1)].tolist())
+    row = g[0].cpu().numpy()
+    assert O.check_topk_sign_row(row, K, idx_g, sgn_g) == ""
+    del row
+    vote_o, bad = O.majority_vote(idx_g[None, :], sgn_g[None, :], 1, K, d)
+    assert bad == 0 and int(np.count_nonzero(vote_o)) == K
+
+    chunk = 1 << 28
+    x_o = np.empty(d, np.float32)
+    for lo in range(0, d, chunk):
+        x_o[lo:lo + chunk] = O.apply_vote(x0[lo:lo + chunk].cpu().numpy(), vote_o[lo:lo + chunk], lr)
+
+    def same_x(x_dev, tag):
+        for lo in range(0, d, chunk):
+            assert np.array_equal(u32(x_dev[lo:lo + chunk]), x_o[lo:lo + chunk].view(np.uint32)), \
+                f"{tag}: x differs in [{lo}, {lo + chunk})"
+
+    same_x(x, "step with the message")
+    del idx, sgn
+    x.copy_(x0)
+    S.s3gd_step(x, g, K, lr, ws)                   # the votes-only route
+    code, info = S.s3gd_device_status(ws)
+    assert info[1] == 0
+    same_x(x, "votes-only step")
+    # the three calls, the vote through the int8 buffer
+    x.copy_(x0)
+    vote = torch.empty(d, dtype=torch.int8, device=DEV)
+    idx = torch.from_numpy(idx_g.view(np.int32)).to(DEV)[None, :]
+    sgn = torch.from_numpy(sgn_g.view(np.int32)).to(DEV)[None, :]
+    S.s3gd_majority_vote(idx, sgn, 1, K, d, vote, ws)
+    S.s3gd_apply(x, vote, lr)
+    S.s3gd_device_status(ws)
+    for lo in range(0, d, 1 << 30):
+        assert np.array_equal(vote[lo:lo + (1 << 30)].cpu().numpy(), vote_o[lo:lo + (1 << 30)])
+    same_x(x, "three calls")
+    del vote
+    # K = d: the sign of every entry (Section 3.3, gamma = 1, one worker)
+    x.copy_(x0)
+    S.s3gd_step(x, g, d, lr, ws)
+    S.s3gd_device_status(ws)
+    for lo in range(0, d, 1 << 28):
+        hi = min(d, lo + (1 << 28))
+        neg = (u32(g[0, lo:hi]) >> 31).astype(np.int8)
+        want = O.apply_vote(x0[lo:hi].cpu().numpy(), (1 - 2 * neg).astype(np.int8), lr)
+        assert np.array_equal(bits(x[lo:hi].cpu().numpy()), bits(want)), f"K = d: x differs in [{lo}, {hi})"
 
 
 def test_large_recipe_reduced_64bit_offsets():
@@ -748,6 +824,34 @@ def test_many_workers_plain_and_byte_counters(M, d, K):
     S.s3gd_device_status(ws)
     x_o, _, _, _ = O.randk_step(x.cpu().numpy(), g.cpu().numpy(), Kr, s.lr, 3, 1)
     assert np.array_equal(bits(xr.cpu().numpy()), bits(x_o))
+
+
+@pytest.mark.parametrize("d", [4096, 4097, 4099, 4100, 4101, 4111, 4112, 4113, 4127, 1_000_003])
+def test_update_where_hardly_any_coordinate_is_voted_on(d):
+    """At most one vote per 64 coordinates: the byte counters are then read 32 coordinates at a time.  The last and
+    the first coordinates are voted on, so the words after the last whole group of 16 are exercised too."""
+    M = 3
+    K = max(4, d // 64 // M - 1)
+    gen = torch.Generator(DEV).manual_seed(d)
+    g = torch.randn(M, d, device=DEV, generator=gen)
+    g[:, -3:] = torch.tensor([[50.0, -60.0, 70.0], [-50.0, -60.0, 70.0], [50.0, 60.0, -70.0]], device=DEV)
+    g[:, :2] = torch.tensor([[-80.0, 90.0], [-80.0, -90.0], [80.0, -90.0]], device=DEV)
+    x = torch.randn(d, device=DEV, generator=gen)
+    assert M * K <= d // 64
+    check_all(g, x, K, 0.25, tag=f"sparse votes d={d}")
+    # the same through the exchange call (message in, x out) and with x off its 16-byte alignment
+    idx_o, sgn_o = O.topk_sign(g.cpu().numpy(), K)
+    vote_o, _ = O.majority_vote(idx_o, sgn_o, M, K, d)
+    x_o = O.apply_vote(x.cpu().numpy(), vote_o, 0.25)
+    msg = torch.from_numpy(np.concatenate([idx_o.ravel(), sgn_o.ravel()]).view(np.int32)).to(DEV)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    for off in (0, 1):
+        xb = torch.zeros(d + 4, device=DEV)
+        xv = xb[off:off + d]
+        xv.copy_(x)
+        S.s3gd_vote_apply(xv, msg, 1, msg.numel(), M, K, 0.25, ws)
+        S.s3gd_device_status(ws)
+        assert np.array_equal(bits(xv.cpu().numpy()), bits(x_o)), f"vote_apply d={d} offset {off}"
 
 
 def test_majority_vote_semantics_and_range_flag():
