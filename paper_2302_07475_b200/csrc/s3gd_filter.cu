@@ -25,7 +25,6 @@ __device__ __forceinline__ uint32_t mix32(uint32_t v) {   // integer finaliser, 
 // no more) spread evenly over the row with a hashed offset inside each stride, then
 // tau_lo = lower edge of the highest bin b with (#sampled >= b) >= j_rank.
 constexpr int kChunk = 32;
-constexpr int kSampleUnroll = 16;
 
 // The kernel also resets the row's selection state, its radix histogram and (block 0) the
 // status words, so that no separate initialisation launch is needed on this route.
@@ -68,41 +67,21 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   for (uint32_t b = tid; b < (uint32_t)kHistBins; b += 1024) hist[(uint64_t)row * kHistBins + b] = 0u;
   for (uint32_t b = tid; b < (uint32_t)kSampleBins; b += 1024) s_hist[b] = 0u;
   __syncthreads();
-  // every sampled entry of the row, in the scalar form (short rows, and the error-compensated step,
-  // whose row is formed on the fly from two buffers)
+  // every sampled entry of the row; with error memory the row is formed on the fly from the two buffers.
+  // A short row is inspected whole:
   auto visit_samples = [&](auto&& visit) {
-    if (stride == 0) {                            // short row: every entry is inspected
-      for (uint32_t e = tid; e < n_sample; e += 1024) visit(kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e]);
-      return;
-    }
-    const uint32_t n_chunks = n_sample / kChunk;  // chunk c starts in [c*stride, (c+1)*stride - 32]
-    for (uint32_t c0 = warp; c0 < n_chunks; c0 += 32 * kSampleUnroll) {
-      uint32_t v[kSampleUnroll];
-#pragma unroll
-      for (int u = 0; u < kSampleUnroll; ++u) {
-        const uint32_t c = c0 + 32 * u;
-        if (c < n_chunks) {
-          // offset inside the stride: hash scaled into [0, stride - 31) by a multiply-high (no division)
-          const uint64_t pos = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk - 1)) + lane;
-          v[u] = __ldg(rowp + pos);
-          if (kEF) v[u] = ef_value(v[u], __ldg(errp + pos), eta);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < kSampleUnroll; ++u)
-        if (c0 + 32 * u < n_chunks) visit(v[u]);
-    }
+    for (uint32_t e = tid; e < n_sample; e += 1024) visit(kEF ? ef_value(rowp[e], errp[e], eta) : rowp[e]);
   };
-  if (stride == 0 || kEF) {
-    visit_samples([&](uint32_t b) { atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u); });
-  } else {
-    // chunk c: 32 neighbours starting in [c*stride, (c+1)*stride - 32], on a 16-byte boundary so that a
-    // lane reads four of them at once; eight lanes per chunk, four chunks per warp and load
+  // The long-row form: chunk c is 32 neighbours starting in [c*stride, (c+1)*stride - 32], on a 16-byte boundary
+  // so that a lane reads four of them at once; eight lanes per chunk, four chunks per warp and load.  (The
+  // error memory's rows have the gradient rows' phase within 16 bytes: the host checks.)
+  auto visit_samples_vec = [&](auto&& visit) {
     const uint32_t n_chunks = n_sample / kChunk;
     const uint32_t a4 = (uint32_t)(reinterpret_cast<uintptr_t>(rowp) >> 2) & 3u;     // the row's phase within 16 bytes
-    constexpr int kVecUnroll = 8;
+    constexpr int kVecUnroll = kEF ? 4 : 8;
     for (uint32_t c0 = warp * 4 + (lane >> 3); c0 < n_chunks; c0 += 32 * 4 * kVecUnroll) {
       uint4 v[kVecUnroll];
+      float4 e[kEF ? kVecUnroll : 1];
 #pragma unroll
       for (int u = 0; u < kVecUnroll; ++u) {
         const uint32_t c = c0 + 32 * 4 * u;
@@ -112,19 +91,26 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
           const uint64_t p = (uint64_t)c * stride + __umulhi(mix32(c), stride - (kChunk + 2));
           const uint64_t pos = ((p + a4 + 3u) & ~(uint64_t)3u) - a4 + (lane & 7u) * 4u;
           v[u] = ld_stream_v4(rowp + pos);
+          if (kEF) e[u] = __ldg(reinterpret_cast<const float4*>(errp + pos));
         }
       }
 #pragma unroll
       for (int u = 0; u < kVecUnroll; ++u) {
         if (c0 + 32 * 4 * u < n_chunks) {
-          atomicAdd(&s_hist[(v[u].x & kAbsMask) >> 16], 1u);
-          atomicAdd(&s_hist[(v[u].y & kAbsMask) >> 16], 1u);
-          atomicAdd(&s_hist[(v[u].z & kAbsMask) >> 16], 1u);
-          atomicAdd(&s_hist[(v[u].w & kAbsMask) >> 16], 1u);
+          if (kEF) {
+            v[u].x = ef_value(v[u].x, e[u].x, eta); v[u].y = ef_value(v[u].y, e[u].y, eta);
+            v[u].z = ef_value(v[u].z, e[u].z, eta); v[u].w = ef_value(v[u].w, e[u].w, eta);
+          }
+          visit(v[u].x); visit(v[u].y); visit(v[u].z); visit(v[u].w);
         }
       }
     }
-  }
+  };
+  auto visit_all = [&](auto&& visit) {
+    if (stride == 0) visit_samples(visit);
+    else visit_samples_vec(visit);
+  };
+  visit_all([&](uint32_t b) { atomicAdd(&s_hist[(b & kAbsMask) >> 16], 1u); });
   __syncthreads();
 
   // warp w owns bins [1024 w, 1024 w + 1024): conflict-free strided reads
@@ -203,7 +189,7 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
     const uint32_t bin = s_fine[0], above_bin = s_fine[1];
     for (uint32_t b = tid; b < 256u; b += 1024) s_hist[b] = 0u;          // (both searches are past the barrier)
     __syncthreads();
-    visit_samples([&](uint32_t b) {
+    visit_all([&](uint32_t b) {
       const uint32_t key = b & kAbsMask;
       if ((key >> 16) == bin) atomicAdd(&s_hist[(key >> 8) & 0xFFu], 1u);
     });

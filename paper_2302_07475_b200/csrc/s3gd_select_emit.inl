@@ -480,14 +480,10 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
   // Rows whose candidates fit one SM are finished by one CTA each; if only the votes are wanted and a
   // typical row needs the shared memory of up to four SMs, by a cluster of CTAs each.
   const bool votes_only = counter != nullptr && out_idx == nullptr && out_signbits == nullptr;
-  // With error compensation the residuals pile up just below the threshold, so rows run above the
-  // sampling estimate: take the next larger on-chip form there.
-  const uint32_t expect = err_to_clear ? 2u * L.typical_cand : L.typical_cand;
+  // (With error compensation the residuals pile up just below the threshold; the sampler places tau_lo
+  // inside its histogram bin there, which keeps the rows at the sampling estimate.)
   uint32_t cluster = 0u;
-  if (use_filter && votes_only) {
-    if (!fits_single_cta(expect)) cluster = cluster_size_for(expect);
-    if (cluster == 0u && !fits_single_cta(L.typical_cand)) cluster = cluster_size_for(L.typical_cand);
-  }
+  if (use_filter && votes_only && !fits_single_cta(L.typical_cand)) cluster = cluster_size_for(L.typical_cand);
   // If a row's candidates are expected to fit an on-chip selection, the general passes only serve the
   // odd row that did not fit or fell back to the whole-row route.
   const bool only_fallback = use_filter && (fits_single_cta(L.typical_cand) || cluster != 0u);

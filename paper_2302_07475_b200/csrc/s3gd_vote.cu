@@ -263,6 +263,43 @@ __global__ void __launch_bounds__(256) apply_momentum_kernel(float* __restrict__
   }
 }
 
+// Four coordinates per thread: one word of byte counters (or four int32 counters, or four int8 votes:
+// kSource 0 / 1 / 2), x and v as float4.  x and v 16-byte aligned, counters 16-byte aligned, votes 4-byte aligned.
+template <int kSource>
+__global__ void __launch_bounds__(256) momentum_v4_kernel(const void* __restrict__ src, float4* __restrict__ x4,
+                                                          float4* __restrict__ v4, uint64_t n4, float mu, float lr,
+                                                          uint32_t* __restrict__ opt_vote4) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    int c[4];
+    if (kSource == 0) {
+      const uint32_t w = static_cast<const uint32_t*>(src)[i];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) c[q] = (int)((w >> (8 * q)) & 0xFFu) - 128;
+    } else if (kSource == 1) {
+      const int4 cc = static_cast<const int4*>(src)[i];
+      c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w;
+    } else {
+      const uint32_t w = static_cast<const uint32_t*>(src)[i];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) c[q] = (int)(int8_t)((w >> (8 * q)) & 0xFFu);
+    }
+    float4 xv = x4[i], vv = v4[i];
+    momentum_update(xv.x, vv.x, c[0], mu, lr);
+    momentum_update(xv.y, vv.y, c[1], mu, lr);
+    momentum_update(xv.z, vv.z, c[2], mu, lr);
+    momentum_update(xv.w, vv.w, c[3], mu, lr);
+    x4[i] = xv;
+    v4[i] = vv;
+    if (kSource != 2 && opt_vote4) {
+      uint32_t pk = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) pk |= (uint32_t)(uint8_t)(int8_t)((c[q] > 0) - (c[q] < 0)) << (8 * q);
+      opt_vote4[i] = pk;
+    }
+  }
+}
+
 inline unsigned grid_for(uint64_t items, int per_block, int max_blocks) {
   uint64_t b = (items + per_block - 1) / per_block;
   if (b < 1) b = 1;
@@ -350,15 +387,47 @@ cudaError_t launch_ef_accumulate(float* err, const float* grads, float eta, uint
 
 cudaError_t launch_counter_apply_momentum(const int32_t* counter, bool packed, float* x, float* v, uint64_t d, float mu,
                                           float lr, int8_t* opt_vote, cudaStream_t st) {
-  if (packed) counter_apply_momentum_kernel<true><<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
-  else counter_apply_momentum_kernel<false><<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, x, v, d, mu, lr, opt_vote);
+  // dense over d (v decays everywhere): four coordinates per thread and one thread per group where the
+  // alignment allows, the scalar form for what is left over
+  uint64_t done = 0;
+  if (d >= 4 && aligned(x, 16) && aligned(v, 16) && aligned(counter, 16) && (opt_vote == nullptr || aligned(opt_vote, 4))) {
+    const uint64_t n4 = d / 4;
+    const unsigned grid = grid_for(n4, 256, 0x7FFFFFFF);
+    if (packed)
+      momentum_v4_kernel<0><<<grid, 256, 0, st>>>(counter, reinterpret_cast<float4*>(x), reinterpret_cast<float4*>(v), n4,
+                                                  mu, lr, reinterpret_cast<uint32_t*>(opt_vote));
+    else
+      momentum_v4_kernel<1><<<grid, 256, 0, st>>>(counter, reinterpret_cast<float4*>(x), reinterpret_cast<float4*>(v), n4,
+                                                  mu, lr, reinterpret_cast<uint32_t*>(opt_vote));
+    count_launch();
+    done = n4 * 4;
+    if (done == d) return cudaGetLastError();
+  }
+  const uint64_t rest = d - done;
+  int8_t* ov = opt_vote ? opt_vote + done : nullptr;
+  if (packed)
+    counter_apply_momentum_kernel<true><<<grid_for(rest, 256, sm_count() * 16), 256, 0, st>>>(
+        reinterpret_cast<const int32_t*>(reinterpret_cast<const uint8_t*>(counter) + done), x + done, v + done, rest, mu, lr, ov);
+  else
+    counter_apply_momentum_kernel<false><<<grid_for(rest, 256, sm_count() * 16), 256, 0, st>>>(counter + done, x + done,
+                                                                                             v + done, rest, mu, lr, ov);
   count_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_apply_momentum(float* x, float* v, const int8_t* vote, uint64_t d, float mu, float lr,
                                   cudaStream_t st) {
-  apply_momentum_kernel<<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(x, v, vote, d, mu, lr);
+  uint64_t done = 0;
+  if (d >= 4 && aligned(x, 16) && aligned(v, 16) && aligned(vote, 4)) {
+    const uint64_t n4 = d / 4;
+    momentum_v4_kernel<2><<<grid_for(n4, 256, 0x7FFFFFFF), 256, 0, st>>>(vote, reinterpret_cast<float4*>(x),
+                                                                        reinterpret_cast<float4*>(v), n4, mu, lr, nullptr);
+    count_launch();
+    done = n4 * 4;
+    if (done == d) return cudaGetLastError();
+  }
+  apply_momentum_kernel<<<grid_for(d - done, 256, sm_count() * 16), 256, 0, st>>>(x + done, v + done, vote + done, d - done,
+                                                                                mu, lr);
   count_launch();
   return cudaGetLastError();
 }

@@ -718,16 +718,38 @@ def test_momentum_without_error_memory_over_steps(K):
         assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)), f"step {step}: x differs"
 
 
-def test_unfused_momentum_update():
-    d = 100_003
-    gen = torch.Generator(DEV).manual_seed(5)
-    x = torch.randn(d, device=DEV, generator=gen)
-    v = torch.randn(d, device=DEV, generator=gen)
-    vote = torch.randint(-1, 2, (d,), device=DEV, generator=gen, dtype=torch.int8)
+@pytest.mark.parametrize("d", [1, 3, 4, 5, 4096, 100_003])
+@pytest.mark.parametrize("x_off,v_off,vote_off", [(0, 0, 0), (1, 0, 0), (0, 2, 0), (0, 0, 1), (3, 3, 3)])
+def test_unfused_momentum_update(d, x_off, v_off, vote_off):
+    """s3gd_apply_momentum for lengths around the four-coordinate groups and for buffers off their alignment."""
+    gen = torch.Generator(DEV).manual_seed(5 + d)
+    x = torch.randn(d + 4, device=DEV, generator=gen)[x_off:x_off + d]
+    v = torch.randn(d + 4, device=DEV, generator=gen)[v_off:v_off + d]
+    vote = torch.randint(-1, 2, (d + 4,), device=DEV, generator=gen, dtype=torch.int8)[vote_off:vote_off + d]
     x_o, v_o = O.apply_vote_momentum(x.cpu().numpy(), v.cpu().numpy(), vote.cpu().numpy(), 0.9, 1e-3)
     S.s3gd_apply_momentum(x, v, vote, 0.9, 1e-3)
     torch.cuda.synchronize()
     assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)) and np.array_equal(bits(v.cpu().numpy()), bits(v_o))
+
+
+@pytest.mark.parametrize("M", [5, 130])
+@pytest.mark.parametrize("d,x_off,v_off", [(40_000, 0, 0), (40_003, 0, 0), (40_003, 1, 0), (40_002, 0, 3)])
+def test_fused_momentum_update_alignments(M, d, x_off, v_off):
+    """The momentum update at the end of the fused step: byte and int32 counters, vote output, buffers off alignment."""
+    K = 400
+    gen = torch.Generator(DEV).manual_seed(d + M)
+    g = torch.randn(M, d, device=DEV, generator=gen)
+    x = torch.randn(d + 4, device=DEV, generator=gen)[x_off:x_off + d]
+    v = torch.randn(d + 4, device=DEV, generator=gen)[v_off:v_off + d]
+    vote = torch.full((d,), 77, dtype=torch.int8, device=DEV)
+    x_o, v_o = x.cpu().numpy(), v.cpu().numpy()
+    _, _, _, vote_o = O.step(x_o, g.cpu().numpy(), K, 0.01)
+    x_o, v_o = O.apply_vote_momentum(x_o, v_o, vote_o, 0.5, 0.01)
+    ws = S.alloc_workspace(M, d, K, DEV)
+    S.s3gd_step_ex(x, g, K, 0.01, ws, v=v, mu=0.5, opt_vote=vote)
+    S.s3gd_device_status(ws)
+    assert np.array_equal(vote.cpu().numpy(), vote_o)
+    assert np.array_equal(bits(v.cpu().numpy()), bits(v_o)) and np.array_equal(bits(x.cpu().numpy()), bits(x_o))
 
 
 # ------------------------------------------------ random-K variant (Section 3.4, Algorithm 2)
