@@ -214,6 +214,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   __shared__ uint32_t s_hist[kHistBins];
   __shared__ uint32_t s_warp[kSmallWarps];
   __shared__ uint32_t s_sel[2];
+  __shared__ uint32_t s_first[kOrdered ? kSmallThreads : 1];   // first chunk of each tile of a layout round
   const uint32_t row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, lt = lanemask_lt();
   const RowState rs = rows[row];
   if (kBin ? rs.done != kRowBin : !row_uses_candidates(rs, o.K, cap)) return;
@@ -245,48 +246,71 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   } else {
     // ---- bring the candidates on chip in index order: the filter stored them tile by tile, each
     // tile's segment wherever its claim landed; laying the segments out in tile order sorts them.
-    // A warp takes 32 consecutive tiles per step (one per lane for the bookkeeping), then copies
-    // their segments with all lanes, several segments' loads in flight before the first store.
+    // 1024 tiles per round (one per thread for the bookkeeping).  The round's segments are cut into
+    // chunks of up to 32 entries -- a tile with c entries has ceil(c / 32), an empty one none -- and the
+    // chunks are dealt to the warps in turn, eight chunks' loads in flight per warp before the first
+    // store: gradients with layer-wise scales put hundreds of candidates into the tiles of a few layers
+    // and none into most, and a division by tiles left most warps waiting for a few.
     {
+      static_assert(kHistBins >= 2 * kSmallThreads, "two tables of the layout live in the histogram's words");
+      uint32_t* s_src = s_hist;                      // (the histogram is not in use yet)
+      uint32_t* s_dst = s_hist + kSmallThreads;
       const uint32_t warp = tid >> 5;
       uint32_t carry = 0;
       for (uint32_t base = 0; base < n_tiles; base += kSmallThreads) {
         const uint32_t t = base + tid;
         const uint2 sg = t < n_tiles ? seg[(uint64_t)row * n_tiles + t] : make_uint2(0u, 0u);
-        uint32_t total;
+        uint32_t total, total_chunks;
         const uint32_t dst = carry + block_scan_excl_1024(sg.y, s_warp, &total);
-        carry += total;
-        const uint32_t longest = __reduce_max_sync(0xFFFFFFFFu, sg.y);
-        if (longest == 0u) continue;                 // warp-uniform
-        if (longest <= 32u) {
-          constexpr int kBatch = 8;
-  #pragma unroll 1
-          for (int j0 = 0; j0 < 32; j0 += kBatch) {
+        const uint32_t first_chunk = block_scan_excl_1024((sg.y + 31u) >> 5, s_warp, &total_chunks);
+        const uint32_t end = carry + total;          // where the round's last segment ends
+        carry = end;
+        s_src[tid] = sg.x;
+        s_dst[tid] = dst;
+        s_first[tid] = first_chunk;
+        __syncthreads();
+        // a warp takes 32 chunks at a time, one per lane for the lookup: the chunk's tile is the last one whose
+        // first chunk is <= k (first_chunk does not decrease; an empty tile shares its value with the next one)
+        constexpr int kBatch = 8;
+#pragma unroll 1
+        for (uint32_t k0 = warp * 32u; k0 < total_chunks; k0 += kSmallWarps * 32u) {   // warp-uniform
+          const uint32_t k = k0 + lane;
+          uint32_t my_d0 = 0, my_cnt = 0, my_src = 0, my_off = 0;
+          if (k < total_chunks) {
+            uint32_t lo = 0, len = kSmallThreads;        // invariant: s_first[lo] <= k
+#pragma unroll
+            for (int it = 0; it < 10; ++it) {
+              len >>= 1;
+              if (s_first[lo + len] <= k) lo += len;
+            }
+            my_d0 = s_dst[lo];
+            my_cnt = (lo + 1u < (uint32_t)kSmallThreads ? s_dst[lo + 1u] : end) - my_d0;
+            my_src = s_src[lo];
+            my_off = (k - s_first[lo]) * 32u;
+          }
+          const uint32_t n_here = total_chunks - k0 < 32u ? total_chunks - k0 : 32u;
+#pragma unroll 1
+          for (uint32_t j0 = 0; j0 < n_here; j0 += kBatch) {
             uint2 e[kBatch];
             uint32_t at[kBatch];
-  #pragma unroll
+#pragma unroll
             for (int j = 0; j < kBatch; ++j) {
-              const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j0 + j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j0 + j);
-              const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j0 + j);
-              at[j] = lane < cnt ? d0 + lane : 0xFFFFFFFFu;
-              if (lane < cnt) e[j] = c[src + lane];
+              const uint32_t jj = j0 + j;                  // (a lane beyond n_here holds zeros: nothing to copy)
+              const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, my_d0, jj & 31u), cnt = __shfl_sync(0xFFFFFFFFu, my_cnt, jj & 31u);
+              const uint32_t src = __shfl_sync(0xFFFFFFFFu, my_src, jj & 31u);
+              const uint32_t i = __shfl_sync(0xFFFFFFFFu, my_off, jj & 31u) + lane;
+              at[j] = 0xFFFFFFFFu;
+              if (jj < n_here && i < cnt) {
+                at[j] = d0 + i;
+                e[j] = c[src + i];
+              }
             }
-  #pragma unroll
+#pragma unroll
             for (int j = 0; j < kBatch; ++j)
               if (at[j] != 0xFFFFFFFFu) { s_bits[at[j]] = e[j].x; s_idx[at[j]] = e[j].y; }
           }
-        } else {                                     // some long segment: one tile after the other
-          for (int j = 0; j < 32; ++j) {
-            const uint32_t src = __shfl_sync(0xFFFFFFFFu, sg.x, j), cnt = __shfl_sync(0xFFFFFFFFu, sg.y, j);
-            const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, dst, j);
-            for (uint32_t i = lane; i < cnt; i += 32) {
-              const uint2 e = c[src + i];
-              s_bits[d0 + i] = e.x;
-              s_idx[d0 + i] = e.y;
-            }
-          }
         }
-        (void)warp;
+        __syncthreads();                             // the three tables are rewritten by the next round
       }
     }
   }
@@ -474,6 +498,13 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   // the number of block-wide scans, and with it of warp shuffles, small.)
   constexpr int kPer = 16;
   uint32_t carry_eq = 0, carry_out = 0;
+  // the row's sign words are put together in shared memory (the histogram's words are free again;
+  // K <= n <= 27k entries are at most 848 words) and written out whole at the end
+  const bool sign_on_chip = o.signbits != nullptr && o.words <= (uint32_t)kHistBins;
+  if (sign_on_chip) {
+    for (uint32_t w = tid; w < o.words; w += kSmallThreads) s_hist[w] = 0u;
+    __syncthreads();
+  }
   for (uint32_t base = 0; base < n; base += kSmallThreads * kPer) {
     const uint32_t i0 = base + tid * kPer;
     uint32_t bits[kPer], eqf = 0, inf = 0;
@@ -486,19 +517,19 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
     }
     uint32_t tot_eq, tot_sel;
     const uint32_t tie0 = carry_eq + block_scan_excl_1024(__popc(eqf), s_warp, &tot_eq);
-    uint32_t self = 0;
+    uint32_t self = 0, tie = tie0;
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
       const uint32_t key = bits[q] & kAbsMask;
-      const bool keep = (inf >> q & 1u) &&
-                        (key > tau || ((eqf >> q & 1u) && tie0 + __popc(eqf & ((1u << q) - 1u)) < take));
+      const uint32_t is_eq = eqf >> q & 1u;
+      const bool keep = (inf >> q & 1u) && (key > tau || (is_eq && tie < take));
+      tie += is_eq;
       self |= (uint32_t)keep << q;
     }
-    const uint32_t pos0 = carry_out + block_scan_excl_1024(__popc(self), s_warp, &tot_sel);
+    uint32_t pos = carry_out + block_scan_excl_1024(__popc(self), s_warp, &tot_sel);
 #pragma unroll
     for (int q = 0; q < kPer; ++q) {
       if (self >> q & 1u) {
-        const uint32_t pos = pos0 + __popc(self & ((1u << q) - 1u));
         if (pos < o.K) {
           const uint32_t idx = s_idx[i0 + q];
           const uint32_t neg = bits[q] >> 31;
@@ -506,12 +537,20 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
           if (o.counter) add_vote(o.counter, o.packed, idx, neg);
           if (o.err) o.err[(uint64_t)row * o.d + idx] = 0.f;
           // sign bits only when the message is asked for: one atomic per negative entry
-          if (o.signbits && neg) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
+          if (neg) {
+            if (sign_on_chip) atomicOr(&s_hist[pos >> 5], 1u << (pos & 31));
+            else if (o.signbits) atomicOr(o.signbits + (uint64_t)row * o.words + (pos >> 5), 1u << (pos & 31));
+          }
         }
+        ++pos;
       }
     }
     carry_eq += tot_eq;
     carry_out += tot_sel;
+  }
+  if (sign_on_chip) {
+    __syncthreads();
+    for (uint32_t w = tid; w < o.words; w += kSmallThreads) o.signbits[(uint64_t)row * o.words + w] = s_hist[w];
   }
   if (tid == 0) {
     rows[row].tau = tau;

@@ -67,6 +67,19 @@ __global__ void __launch_bounds__(256) vote_scatter_kernel(const uint32_t* __res
   }
 }
 
+__global__ void __launch_bounds__(256) counter_sign_v4_kernel(const int4* __restrict__ counter4, uint64_t n4,
+                                                              uint32_t* __restrict__ vote4) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const int4 c = counter4[i];
+    const int s[4] = {(c.x > 0) - (c.x < 0), (c.y > 0) - (c.y < 0), (c.z > 0) - (c.z < 0), (c.w > 0) - (c.w < 0)};
+    uint32_t pk = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) pk |= (uint32_t)(uint8_t)(int8_t)s[q] << (8 * q);
+    vote4[i] = pk;
+  }
+}
+
 __global__ void __launch_bounds__(256) counter_sign_kernel(const int32_t* __restrict__ counter, uint64_t d,
                                                            int8_t* __restrict__ vote) {
   uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
@@ -314,7 +327,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 cudaError_t launch_apply(float* x, const int8_t* vote, uint64_t d, float lr, cudaStream_t st) {
   if (aligned(x, 16) && aligned(vote, 16) && d >= 16) {
     uint64_t n16 = d / 16;
-    apply_kernel_v16<<<grid_for(n16, 256, sm_count() * 8), 256, 0, st>>>(x, vote, n16, lr);
+    apply_kernel_v16<<<grid_for(n16, 256, 0x7FFFFFFF), 256, 0, st>>>(x, vote, n16, lr);
     count_launch();
     uint64_t done = n16 * 16;
     if (done < d) apply_kernel<<<1, 256, 0, st>>>(x + done, vote + done, d - done, lr);
@@ -336,7 +349,16 @@ cudaError_t launch_vote_scatter(const uint32_t* idx, const uint32_t* signbits, i
 }
 
 cudaError_t launch_counter_sign(const int32_t* counter, uint64_t d, int8_t* vote, cudaStream_t st) {
-  counter_sign_kernel<<<grid_for(d, 256, sm_count() * 16), 256, 0, st>>>(counter, d, vote);
+  uint64_t done = 0;
+  if (d >= 4 && aligned(counter, 16) && aligned(vote, 4)) {      // four counters in, one word of votes out
+    const uint64_t n4 = d / 4;
+    counter_sign_v4_kernel<<<grid_for(n4, 256, 0x7FFFFFFF), 256, 0, st>>>(reinterpret_cast<const int4*>(counter), n4,
+                                                                         reinterpret_cast<uint32_t*>(vote));
+    count_launch();
+    done = n4 * 4;
+    if (done == d) return cudaGetLastError();
+  }
+  counter_sign_kernel<<<grid_for(d - done, 256, sm_count() * 16), 256, 0, st>>>(counter + done, d - done, vote + done);
   count_launch();
   return cudaGetLastError();
 }
