@@ -54,6 +54,41 @@ __global__ void __launch_bounds__(256) fill_words_kernel(uint32_t* __restrict__ 
 
 __device__ __forceinline__ uint32_t code_of(int c) { return c > 0 ? 1u : (c < 0 ? 3u : 0u); }   // 00, 01 (+1), 11 (-1)
 
+// Sixteen consecutive sums starting at coordinate i (a multiple of 16), as signed totals.  Whole groups
+// from a 16-byte aligned source are fetched with 16-byte loads; the ragged end and other alignments one by one.
+template <int kKind>   // 0: int32 sums, 1: biased bytes, 2: int8 votes
+__device__ __forceinline__ void load_sixteen(const void* __restrict__ src, uint32_t bias, uint64_t n, uint64_t i,
+                                             bool src_aligned, int (&c)[16]) {
+  if (src_aligned && i + 16 <= n) {
+    if (kKind == 0) {
+      const int4* p = reinterpret_cast<const int4*>(static_cast<const int32_t*>(src) + i);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const int4 v = p[g];
+        c[4 * g] = v.x; c[4 * g + 1] = v.y; c[4 * g + 2] = v.z; c[4 * g + 3] = v.w;
+      }
+    } else {
+      const uint4 v = *reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(src) + i);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const uint32_t b = (w[q >> 2] >> (8 * (q & 3))) & 0xFFu;
+        c[q] = kKind == 1 ? (int)(int8_t)(uint8_t)(b - bias) : (int)(int8_t)(uint8_t)b;
+      }
+    }
+    return;
+  }
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    c[q] = 0;
+    if (i + q < n) {
+      if (kKind == 0) c[q] = static_cast<const int32_t*>(src)[i + q];
+      else if (kKind == 1) c[q] = (int)(int8_t)(uint8_t)(static_cast<const uint8_t*>(src)[i + q] - bias);
+      else c[q] = static_cast<const int8_t*>(src)[i + q];
+    }
+  }
+}
+
 // sixteen coordinates -> one word of two-bit codes.  kBytes: one byte per coordinate holding the
 // sum of `n_summed` biased bytes (each 128 + a partial sum), reduced modulo 256; the total then is
 // (byte - 128 * n_summed) as a signed byte.  Otherwise int32 sums (or int8 votes, kVotes).
@@ -62,18 +97,13 @@ __global__ void __launch_bounds__(256) encode2_kernel(const void* __restrict__ s
                                                       uint32_t* __restrict__ out) {
   const uint64_t n_words = (n + 15) / 16;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const bool src_aligned = (reinterpret_cast<uintptr_t>(src) & 15u) == 0u;
   for (uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += stride) {
+    int c[16];
+    load_sixteen<kKind>(src, bias, n, w * 16, src_aligned, c);
     uint32_t word = 0;
 #pragma unroll
-    for (int q = 0; q < 16; ++q) {
-      const uint64_t i = w * 16 + q;
-      if (i >= n) break;
-      int c;
-      if (kKind == 0) c = static_cast<const int32_t*>(src)[i];
-      else if (kKind == 1) c = (int)(int8_t)(uint8_t)(static_cast<const uint8_t*>(src)[i] - bias);
-      else c = static_cast<const int8_t*>(src)[i];
-      word |= code_of(c) << (2 * q);
-    }
+    for (int q = 0; q < 16; ++q) word |= code_of(c[q]) << (2 * q);      // (beyond n: 0, the code of "no vote")
     out[w] = word;
   }
 }
@@ -110,28 +140,18 @@ constexpr int kSparseThreads = 256;
 constexpr int kSparsePer = 16;                                     // consecutive coordinates per thread
 constexpr int kSparseBlock = kSparseThreads * kSparsePer;          // coordinates per block
 
-template <int kKind>
-__device__ __forceinline__ int vote_of(const void* __restrict__ src, uint32_t bias, uint64_t i) {
-  int c;
-  if (kKind == 0) c = static_cast<const int32_t*>(src)[i];
-  else if (kKind == 1) c = (int)(int8_t)(uint8_t)(static_cast<const uint8_t*>(src)[i] - bias);
-  else c = static_cast<const int8_t*>(src)[i];
-  return (c > 0) - (c < 0);
-}
-
 // bit q of the results: coordinate first + q has a non-zero vote / a negative one
 template <int kKind>
 __device__ __forceinline__ void thread_votes(const void* __restrict__ src, uint32_t bias, uint64_t n, uint64_t first,
                                              uint32_t* moved, uint32_t* negative) {
+  static_assert(kSparsePer == 16, "a thread's coordinates are one group of load_sixteen");
+  int c[16];
+  load_sixteen<kKind>(src, bias, n, first, (reinterpret_cast<uintptr_t>(src) & 15u) == 0u, c);
   uint32_t mv = 0, ng = 0;
 #pragma unroll
   for (int q = 0; q < kSparsePer; ++q) {
-    const uint64_t i = first + q;
-    if (i < n) {
-      const int v = vote_of<kKind>(src, bias, i);
-      mv |= (uint32_t)(v != 0) << q;
-      ng |= (uint32_t)(v < 0) << q;
-    }
+    mv |= (uint32_t)(c[q] != 0) << q;                 // (beyond n: 0)
+    ng |= (uint32_t)(c[q] < 0) << q;
   }
   *moved = mv; *negative = ng;
 }
@@ -307,7 +327,7 @@ s3gd_status s3gd_encode_vote2(const void* src, int src_kind, uint32_t n_summed, 
     return S3GD_ERR_INVALID_ARG;
   if (src_kind == 0 && !aligned(src, 4)) return S3GD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const unsigned grid = grid_for((n + 15) / 16, 256, sm_count() * 8);
+  const unsigned grid = grid_for((n + 15) / 16, 256, 0x7FFFFFFF);     // one thread per word: blocks that come and go
   const uint32_t bias = (128u * n_summed) & 0xFFu;
   if (src_kind == 0) encode2_kernel<0><<<grid, 256, 0, st>>>(src, 0u, n, out_words);
   else if (src_kind == 1) encode2_kernel<1><<<grid, 256, 0, st>>>(src, bias, n, out_words);
@@ -321,7 +341,7 @@ s3gd_status s3gd_apply_vote2(float* x, const uint32_t* words, uint64_t d, float 
   if (x == nullptr || words == nullptr || d == 0 || d >= (1ull << 32) || !aligned(x, 4) || !aligned(words, 4))
     return S3GD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  apply2_kernel<<<grid_for((d + 15) / 16, 256, sm_count() * 8), 256, 0, st>>>(x, words, d, lr, opt_vote);
+  apply2_kernel<<<grid_for((d + 15) / 16, 256, 0x7FFFFFFF), 256, 0, st>>>(x, words, d, lr, opt_vote);
   if (cudaGetLastError() != cudaSuccess) return S3GD_ERR_CUDA;
   count_launch();
   return S3GD_OK;
