@@ -848,6 +848,17 @@ def test_many_workers_plain_and_byte_counters(M, d, K):
     assert np.array_equal(bits(xr.cpu().numpy()), bits(x_o))
 
 
+@pytest.mark.parametrize("d,K", [(257, 3), (130, 130), (8_201, 33)])
+def test_most_workers_the_interface_accepts(d, K):
+    """M = 65535 rows (the limit: a grid dimension of several kernels): the three routes and K = d, int32 counters."""
+    M = 65_535
+    gen = torch.Generator(DEV).manual_seed(d)
+    g = torch.randn(M, d, device=DEV, generator=gen)
+    g[:, 1] = 50.0; g[:, d - 1] = -50.0                         # unanimous: the counts reach +M and -M
+    x = torch.randn(d, device=DEV, generator=gen)
+    check_all(g, x, K, 0.125, oracle_topk=O.topk_sign_threshold, tag=f"M={M} d={d} K={K}")
+
+
 @pytest.mark.parametrize("d", [4096, 4097, 4099, 4100, 4101, 4111, 4112, 4113, 4127, 1_000_003])
 def test_update_where_hardly_any_coordinate_is_voted_on(d):
     """At most one vote per 64 coordinates: the byte counters are then read 32 coordinates at a time.  The last and
