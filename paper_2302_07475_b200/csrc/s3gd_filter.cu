@@ -241,7 +241,7 @@ constexpr int kWarpStage = 64;                 // survivors a warp can stage per
 
 // magnitude >= tau_lo, decided on the float value: |x| < tau is false for NaN, whose bit
 // pattern is above every threshold, so !(|x| < tau) agrees with the unsigned compare of the
-// sign-less bit patterns for every input (denormals are not flushed in this build).
+// sign-less bit patterns for every input (the library is compiled without flush-to-zero: denormals compare as they are).
 __device__ __forceinline__ bool hit(uint32_t b, float tau) { return !(fabsf(__uint_as_float(b)) < tau); }
 
 template <bool kEF>
