@@ -476,7 +476,7 @@ def test_early_votes_that_are_exactly_the_top_k():
     assert np.array_equal(bits(x.cpu().numpy()), bits(x_o))
 
 
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(200))
 def test_random_shapes_data_and_forced_ranks(seed):
     """A sweep over what the other tests fix by hand: random row lengths beyond the sample size, worker
     counts, K from 1 to d/4, four kinds of data (Gaussian, heavy-tailed with block scales, a handful of
@@ -646,6 +646,64 @@ def test_error_memory_and_momentum_over_steps(K, eta, mu):
             assert np.array_equal(vote.cpu().numpy(), vote_o), f"step {step}: votes differ"
             if K:
                 assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"step {step}: message differs"
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_error_memory_and_momentum(seed):
+    """The sweep of test_random_shapes_data_and_forced_ranks for the extended step: random row lengths, worker counts
+    (both sides of the byte / int32 counter switch), K, eta, mu, data kinds and an error memory that starts
+    non-zero, over three carried steps; x, e, v, votes and the message against the oracle after every step."""
+    rng = np.random.default_rng(7000 + seed)
+    d = int(rng.integers(131_073, 300_000))
+    M = int(rng.choice([1, 2, 5, 9, 130]))
+    K = int(rng.choice([1, 33, d // 1000, d // 100, d // 16, d // 4, d // 3, d]))
+    eta = float(rng.choice([1.0, 1.0, 0.5, 0.0]))
+    mu = [None, 0.9, 0.5][seed % 3]
+    kind = seed % 4
+    lr = 0.03125
+
+    def draw():
+        g = rng.standard_normal((M, d)).astype(np.float32)
+        if kind == 1:
+            g = (rng.standard_t(2.5, (M, d)) * np.repeat(10.0 ** rng.uniform(-3, 0, 16), (d + 15) // 16)[:d]).astype(np.float32)
+        elif kind == 2:
+            g = (rng.choice(np.array([0.0, 0.25, 0.5, 1.0], np.float32), (M, d)) *
+                 rng.choice(np.array([-1.0, 1.0], np.float32), (M, d))).astype(np.float32)
+        elif kind == 3:
+            g[:, d // 3: d // 3 + d // 5] = 2.5
+        return g
+
+    e_o = (0.5 * draw()).astype(np.float32)
+    x_o = rng.standard_normal(d).astype(np.float32)
+    v_o = rng.standard_normal(d).astype(np.float32)
+    err, x = torch.from_numpy(e_o).to(DEV), torch.from_numpy(x_o).to(DEV)
+    v = torch.from_numpy(v_o).to(DEV) if mu is not None else None
+    ws = S.alloc_workspace(M, d, K, DEV)
+    ws.fill_(0x3C)
+    idx = torch.empty((M, K), dtype=torch.int32, device=DEV)
+    sgn = torch.empty((M, S.binding.words(K)), dtype=torch.int32, device=DEV)
+    vote = torch.empty(d, dtype=torch.int8, device=DEV)
+    tag = f"d={d} M={M} K={K} eta={eta} mu={mu} kind={kind}"
+    for step in range(3):
+        g = draw()
+        gt = torch.from_numpy(g).to(DEV)
+        outputs = step != 1
+        if outputs:
+            S.s3gd_step_ex(x, gt, K, lr, ws, err=err, eta=eta, v=v, mu=mu or 0.0, opt_idx=idx, opt_signbits=sgn, opt_vote=vote)
+        else:
+            S.s3gd_step_ex(x, gt, K, lr, ws, err=err, eta=eta, v=v, mu=mu or 0.0)
+        S.s3gd_device_status(ws)
+        xo_plain, e_o, idx_o, sgn_o, vote_o = O.error_feedback_step(x_o, g, e_o, eta, K, lr, topk=O.topk_sign_threshold)
+        if mu is None:
+            x_o = xo_plain
+        else:
+            x_o, v_o = O.apply_vote_momentum(x_o, v_o, vote_o, mu, lr)
+            assert np.array_equal(bits(v.cpu().numpy()), bits(v_o)), f"{tag} step {step}: momentum differs"
+        assert np.array_equal(bits(err.cpu().numpy()), bits(e_o)), f"{tag} step {step}: error memory differs"
+        assert np.array_equal(bits(x.cpu().numpy()), bits(x_o)), f"{tag} step {step}: x differs"
+        if outputs:
+            assert np.array_equal(vote.cpu().numpy(), vote_o), f"{tag} step {step}: votes differ"
+            assert np.array_equal(u32(idx), idx_o) and np.array_equal(u32(sgn), sgn_o), f"{tag} step {step}: message differs"
 
 
 def test_error_memory_in_its_steady_state_keeps_the_single_read_route():
