@@ -244,7 +244,7 @@ def test_longest_row_the_interface_accepts():
     vote is the worker's own TopKSign (Section 3.3, M = 1), which the oracle's vote and update turn into x."""
     if os.environ.get("S3GD_TEST_LARGE") == "0":
         pytest.skip("switched off with S3GD_TEST_LARGE=0")
-    why = _room_for(80e9, 75e9)
+    why = _room_for(100e9, 75e9)
     if why:
         print("longest-row case skipped:", why)
         pytest.skip(why)
@@ -272,22 +272,16 @@ def test_longest_row_the_interface_accepts():
     assert bad == 0 and int(np.count_nonzero(vote_o)) == K
 
     chunk = 1 << 28
-    x_o = np.empty(d, np.float32)
     for lo in range(0, d, chunk):
-        x_o[lo:lo + chunk] = O.apply_vote(x0[lo:lo + chunk].cpu().numpy(), vote_o[lo:lo + chunk], lr)
-
-    def same_x(x_dev, tag):
-        for lo in range(0, d, chunk):
-            assert np.array_equal(u32(x_dev[lo:lo + chunk]), x_o[lo:lo + chunk].view(np.uint32)), \
-                f"{tag}: x differs in [{lo}, {lo + chunk})"
-
-    same_x(x, "step with the message")
+        want = O.apply_vote(x0[lo:lo + chunk].cpu().numpy(), vote_o[lo:lo + chunk], lr)
+        assert np.array_equal(u32(x[lo:lo + chunk]), want.view(np.uint32)), f"step with the message: x differs in [{lo}, {lo + chunk})"
     del idx, sgn
+    x_first = x.clone()                            # equal to the oracle's x: the other routes are compared with it on the device
     x.copy_(x0)
     S.s3gd_step(x, g, K, lr, ws)                   # the votes-only route
     code, info = S.s3gd_device_status(ws)
     assert info[1] == 0
-    same_x(x, "votes-only step")
+    assert torch.equal(x.view(torch.int32), x_first.view(torch.int32)), "votes-only step: x differs"
     # the three calls, the vote through the int8 buffer
     x.copy_(x0)
     vote = torch.empty(d, dtype=torch.int8, device=DEV)
@@ -298,17 +292,20 @@ def test_longest_row_the_interface_accepts():
     S.s3gd_device_status(ws)
     for lo in range(0, d, 1 << 30):
         assert np.array_equal(vote[lo:lo + (1 << 30)].cpu().numpy(), vote_o[lo:lo + (1 << 30)])
-    same_x(x, "three calls")
-    del vote
-    # K = d: the sign of every entry (Section 3.3, gamma = 1, one worker)
+    assert torch.equal(x.view(torch.int32), x_first.view(torch.int32)), "three calls: x differs"
+    del vote, x_first, vote_o
+    # K = d: the sign of every entry (Section 3.3, gamma = 1, one worker); the first chunk, the two around 2^31
+    # and the last one against the oracle's update
     x.copy_(x0)
     S.s3gd_step(x, g, d, lr, ws)
     S.s3gd_device_status(ws)
-    for lo in range(0, d, 1 << 28):
+    for lo in (0, 7 << 28, 8 << 28, 15 << 28):
         hi = min(d, lo + (1 << 28))
         neg = (u32(g[0, lo:hi]) >> 31).astype(np.int8)
         want = O.apply_vote(x0[lo:hi].cpu().numpy(), (1 - 2 * neg).astype(np.int8), lr)
         assert np.array_equal(bits(x[lo:hi].cpu().numpy()), bits(want)), f"K = d: x differs in [{lo}, {hi})"
+    moved = (x != x0)                              # everywhere: every coordinate moves by lr (|x| is far above lr / 2^24)
+    assert bool(moved.all())
 
 
 def test_large_recipe_reduced_64bit_offsets():
