@@ -180,6 +180,9 @@ def test_resnet50_tie_stress_full_size():
 
 
 def _room_for(need_dev, need_host):
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                       # what earlier tests left in torch's cache is free for this one
     free_dev, _ = torch.cuda.mem_get_info()
     if free_dev < need_dev:
         return f"device has {free_dev / 1e9:.0f} GB free, the case needs {need_dev / 1e9:.0f} GB"
