@@ -980,6 +980,52 @@ def test_apply_leaves_unvoted_bits_alone():
         assert np.array_equal(bits(got)[pattern == 0], xb[pattern == 0])
 
 
+def test_host_threads_on_their_own_streams_and_workspaces():
+    """Three host threads step different problems at the same time, each on its own stream with its own
+    workspace (what the interface allows): every result must be the one the oracle gives for that problem."""
+    import threading
+    cases = [(W.spec("resnet18", d=300_007, M=6), 300), (W.spec("resnet50_ties", d=420_001, M=4), 4_200),
+             (W.spec("small_cnn", d=65_536, M=5), 65_536)]
+    jobs = []
+    for s, K in cases:
+        g, x = W.make_grads(s, DEV), W.make_x(s, DEV)
+        x_o, _, _, _ = O.step(x.cpu().numpy(), g.cpu().numpy(), K, s.lr)
+        jobs.append(dict(s=s, K=K, g=g, x=x, x_o=x_o, ws=S.alloc_workspace(s.M, s.d, K, DEV), stream=torch.cuda.Stream(DEV),
+                         out=[], err=None))
+    torch.cuda.synchronize()
+
+    def work(j):
+        try:
+            s, K = j["s"], j["K"]
+            with torch.cuda.stream(j["stream"]):
+                idx = torch.empty((s.M, K), dtype=torch.int32, device=DEV)
+                sgn = torch.empty((s.M, S.binding.words(K)), dtype=torch.int32, device=DEV)
+                vote = torch.empty(s.d, dtype=torch.int8, device=DEV)
+                for it in range(12):
+                    xa = j["x"].clone()
+                    if it % 3 == 2:                          # the three calls now and then
+                        S.s3gd_topk_sign(j["g"], K, idx, sgn, j["ws"])
+                        S.s3gd_majority_vote(idx, sgn, s.M, K, s.d, vote, j["ws"])
+                        S.s3gd_apply(xa, vote, s.lr)
+                    else:
+                        S.s3gd_step(xa, j["g"], K, s.lr, j["ws"])
+                    S.s3gd_device_status(j["ws"])
+                    j["out"].append(xa.cpu().numpy())
+        except Exception as exc:                             # surfaced by the main thread
+            j["err"] = exc
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    for n, j in enumerate(jobs):
+        assert j["err"] is None, f"thread {n}: {j['err']!r}"
+        assert len(j["out"]) == 12
+        for it, xa in enumerate(j["out"]):
+            assert np.array_equal(bits(xa), bits(j["x_o"])), f"thread {n}, iteration {it}: x differs"
+
+
 def test_repeatable():
     s = W.spec("resnet18", d=500_000, M=9)
     g = W.make_grads(s, DEV)
