@@ -37,6 +37,9 @@ NCU_TRAFFIC = {
     "resnet18:11174": {"bytes": int((358.400256e6 + 4.238592e6) * 100 / 8), "digest": "1bed8fb511e91ecb"},
 }
 KERNEL_SOURCES = ("s3gd_filter.cu", "s3gd_tile.cuh", "s3gd_common.cuh")
+# The dominant kernel of every FILTER_EVENTS_EVERY-th timed step is bracketed by two CUDA events (an event
+# record between two kernels costs a microsecond or two of the step, about 5 us per step for the pair).
+FILTER_EVENTS_EVERY = 4
 
 
 def kernel_digest() -> str:
@@ -314,9 +317,10 @@ def acceptance_case(S, W, spec, K, dev, stream, barrier, peak, steps=20, repeats
     for _ in range(3):
         one_step()
     code, info = S.s3gd_device_status(ws)
-    S.s3gd_profile_begin_filter(steps * repeats)
+    n_marked = (steps * repeats + FILTER_EVENTS_EVERY - 1) // FILTER_EVENTS_EVERY
+    S.s3gd_profile_begin_filter_every(n_marked, FILTER_EVENTS_EVERY)
     regions = timed_regions(one_step, steps, repeats, stream, barrier)
-    phases, _ = S.s3gd_profile_end(steps * repeats)
+    phases, _ = S.s3gd_profile_end(n_marked)
     S.s3gd_device_status(ws)
     ms_step = statistics.median(regions) / steps
     filt = [p[1] for p in phases]
@@ -452,12 +456,13 @@ def run_ours(args):
 
     # ---- timed region: device-resident inputs; `repeats` back-to-back regions of `steps` steps, the
     # median region is the reported one.  The library brackets the dominant (filter) kernel of every
-    # timed step with two events; the other phase boundaries are not marked here, because each event
-    # record between two kernels costs a few microseconds of the step.
+    # fourth timed step with two events; the other phase boundaries are not marked here, because each
+    # event record between two kernels costs a microsecond or two of the step.
     sampler = ClockSampler(physical_gpu_index(local_rank)).start()
-    S.s3gd_profile_begin_filter(args.steps * repeats)
+    n_marked = (args.steps * repeats + FILTER_EVENTS_EVERY - 1) // FILTER_EVENTS_EVERY
+    S.s3gd_profile_begin_filter_every(n_marked, FILTER_EVENTS_EVERY)
     regions = timed_regions(one_step, args.steps, repeats, stream, barrier)
-    phases, launches = S.s3gd_profile_end(args.steps * repeats)
+    phases, launches = S.s3gd_profile_end(n_marked)
     clocks = sampler.stop()
     S.s3gd_device_status(ws)
     ms_total = statistics.median(regions)
@@ -559,6 +564,8 @@ def run_ours(args):
                          "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
                          "frac": achieved / peak if achieved else None, "traffic": traffic,
                          "algorithmic_bytes_per_launch": b_grad, "kernel_ms": dom_ms,
+                         "kernel_ms_source": f"CUDA events around every {FILTER_EVENTS_EVERY}th launch inside the timed "
+                                             f"region, {len(kernel_ms)} launches averaged",
                          "dominant_phase": S.binding.PHASES[dominant]},
             "clocks": clocks,
             "gpu_launches": int(round(launches_per_region)),

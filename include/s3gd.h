@@ -353,6 +353,9 @@ S3GD_API s3gd_status s3gd_profile_begin(int max_steps);
  * durations are reported as 0): event records between kernels cost a few microseconds each, so this
  * is the form to leave on while a step is being timed as a whole. */
 S3GD_API s3gd_status s3gd_profile_begin_filter(int max_steps);
+/* The same with only every `every`-th step call recorded (the first one is), at most max_steps of them: a
+ * sample of the filter pass's duration over a long run at 1 / every of the events' cost.  every >= 1. */
+S3GD_API s3gd_status s3gd_profile_begin_filter_every(int max_steps, int every);
 S3GD_API s3gd_status s3gd_profile_end(float* out_ms, int* n_steps, uint64_t* launches);
 
 #ifdef __cplusplus

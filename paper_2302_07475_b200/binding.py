@@ -28,7 +28,8 @@ EXPORTS = ("s3gd_status_string", "s3gd_workspace_bytes", "s3gd_topk_sign", "s3gd
            "s3gd_noalloc_max_d", "s3gd_majority_vote_noalloc", "s3gd_step_ex", "s3gd_apply_momentum",
            "s3gd_randk_sign", "s3gd_step_randk", "s3gd_profile_begin_filter", "s3gd_last_device_status",
            "s3gd_debug_topk_sign", "s3gd_debug_step", "s3gd_vote_apply", "s3gd_vote_counts", "s3gd_encode_vote2",
-           "s3gd_apply_vote2", "s3gd_sparse_workspace_bytes", "s3gd_encode_vote_sparse", "s3gd_apply_vote_sparse")
+           "s3gd_apply_vote2", "s3gd_sparse_workspace_bytes", "s3gd_encode_vote_sparse", "s3gd_apply_vote_sparse",
+           "s3gd_profile_begin_filter_every")
 
 
 class S3gdError(RuntimeError):
@@ -81,6 +82,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.s3gd_apply_momentum.argtypes = [vp, vp, vp, u64, ctypes.c_float, ctypes.c_float, vp]
     lib.s3gd_profile_begin_filter.restype = ctypes.c_int
     lib.s3gd_profile_begin_filter.argtypes = [ctypes.c_int]
+    lib.s3gd_profile_begin_filter_every.restype = ctypes.c_int
+    lib.s3gd_profile_begin_filter_every.argtypes = [ctypes.c_int, ctypes.c_int]
     u32 = ctypes.c_uint32
     lib.s3gd_randk_sign.restype = ctypes.c_int
     lib.s3gd_randk_sign.argtypes = [vp, ctypes.c_int, u64, u64, u32, u32, u32p, u32p, vp, sz, vp]
@@ -340,6 +343,11 @@ def s3gd_profile_begin(max_steps: int) -> None:
 def s3gd_profile_begin_filter(max_steps: int) -> None:
     """As s3gd_profile_begin, but only the filter pass is bracketed by events (the other phases read 0)."""
     _check("s3gd_profile_begin_filter", load().s3gd_profile_begin_filter(int(max_steps)))
+
+
+def s3gd_profile_begin_filter_every(max_steps: int, every: int) -> None:
+    """As s3gd_profile_begin_filter with only every `every`-th step recorded (at most max_steps of them)."""
+    _check("s3gd_profile_begin_filter_every", load().s3gd_profile_begin_filter_every(int(max_steps), int(every)))
 
 
 def s3gd_profile_end(max_steps: int):

@@ -108,17 +108,22 @@ namespace {
 struct Profiler {
   bool on = false;
   bool filter_only = false;           // record only the two marks around the filter pass
-  int max_steps = 0, n_steps = 0;
+  int max_steps = 0, n_steps = 0;     // steps to record at most / recorded so far
+  int every = 1, n_calls = 0;         // every `every`-th step is recorded / steps seen so far
   cudaEvent_t* ev = nullptr;          // kPhaseMarks events per recorded step
 } g_prof;
 std::atomic<unsigned long long> g_launches{0};   // kernels enqueued while a profiling session is open
 }  // namespace
 
 void prof_mark(int phase, cudaStream_t st) {
-  if (!g_prof.on || g_prof.n_steps >= g_prof.max_steps) return;
-  if (!g_prof.filter_only || phase == kPhaseSampled || phase == kPhaseFiltered)
+  if (!g_prof.on) return;
+  const bool recorded = g_prof.n_steps < g_prof.max_steps && g_prof.n_calls % g_prof.every == 0;
+  if (recorded && (!g_prof.filter_only || phase == kPhaseSampled || phase == kPhaseFiltered))
     cudaEventRecord(g_prof.ev[(size_t)g_prof.n_steps * kPhaseMarks + phase], st);
-  if (phase == kPhaseApplied) ++g_prof.n_steps;
+  if (phase == kPhaseApplied) {                  // the last mark of a step
+    if (recorded) ++g_prof.n_steps;
+    ++g_prof.n_calls;
+  }
 }
 
 void count_launch(int n) {
@@ -392,15 +397,16 @@ s3gd_status s3gd_step_randk(float* x, const float* grads, int M, uint64_t d, uin
 }
 
 namespace {
-s3gd_status profile_begin(int max_steps, bool filter_only);
+s3gd_status profile_begin(int max_steps, bool filter_only, int every);
 }
 
-s3gd_status s3gd_profile_begin(int max_steps) { return profile_begin(max_steps, false); }
-s3gd_status s3gd_profile_begin_filter(int max_steps) { return profile_begin(max_steps, true); }
+s3gd_status s3gd_profile_begin(int max_steps) { return profile_begin(max_steps, false, 1); }
+s3gd_status s3gd_profile_begin_filter(int max_steps) { return profile_begin(max_steps, true, 1); }
+s3gd_status s3gd_profile_begin_filter_every(int max_steps, int every) { return profile_begin(max_steps, true, every); }
 
 namespace {
-s3gd_status profile_begin(int max_steps, bool filter_only) {
-  if (max_steps <= 0 || max_steps > (1 << 20) || g_prof.on) return S3GD_ERR_INVALID_ARG;
+s3gd_status profile_begin(int max_steps, bool filter_only, int every) {
+  if (max_steps <= 0 || max_steps > (1 << 20) || every < 1 || g_prof.on) return S3GD_ERR_INVALID_ARG;
   const size_t n = (size_t)max_steps * kPhaseMarks;
   g_prof.ev = new cudaEvent_t[n];
   for (size_t i = 0; i < n; ++i) {
@@ -413,6 +419,8 @@ s3gd_status profile_begin(int max_steps, bool filter_only) {
   }
   g_prof.max_steps = max_steps;
   g_prof.n_steps = 0;
+  g_prof.every = every;
+  g_prof.n_calls = 0;
   g_launches.store(0);
   g_prof.filter_only = filter_only;
   g_prof.on = true;

@@ -1026,6 +1026,42 @@ def test_host_threads_on_their_own_streams_and_workspaces():
             assert np.array_equal(bits(xa), bits(j["x_o"])), f"thread {n}, iteration {it}: x differs"
 
 
+def test_phase_timing_sessions():
+    """The measurement aid: all phases of every step, the filter pass of every step, the filter pass of every
+    second step; the step's result is the same with and without a session open."""
+    s = W.spec("resnet18", d=300_007, M=6)
+    K = 300
+    g, x0 = W.make_grads(s, DEV), W.make_x(s, DEV)
+    ws = S.alloc_workspace(s.M, s.d, K, DEV)
+    ref = x0.clone()
+    S.s3gd_step(ref, g, K, s.lr, ws)
+    S.s3gd_device_status(ws)
+
+    def five_steps():
+        for _ in range(5):
+            x = x0.clone()
+            S.s3gd_step(x, g, K, s.lr, ws)
+            assert torch.equal(x.view(torch.int32), ref.view(torch.int32))
+
+    S.s3gd_profile_begin(8)
+    five_steps()
+    steps, launches = S.s3gd_profile_end(8)
+    assert len(steps) == 5 and launches > 0 and all(p[1] > 0 and p[4] > 0 for p in steps)
+    S.s3gd_profile_begin_filter(3)                      # room for three steps only
+    five_steps()
+    steps, _ = S.s3gd_profile_end(3)
+    assert len(steps) == 3 and all(p[1] > 0 and p[0] == 0 and p[4] == 0 for p in steps)
+    S.s3gd_profile_begin_filter_every(8, 2)             # steps 0, 2 and 4 of the five
+    five_steps()
+    steps, launches_b = S.s3gd_profile_end(8)
+    assert len(steps) == 3 and all(p[1] > 0 for p in steps) and launches_b == launches
+    with pytest.raises(S.S3gdError):
+        S.s3gd_profile_begin_filter_every(8, 0)
+    with pytest.raises(S.S3gdError):
+        S.s3gd_profile_end(1)                           # no session open
+    S.s3gd_device_status(ws)
+
+
 def test_repeatable():
     s = W.spec("resnet18", d=500_000, M=9)
     g = W.make_grads(s, DEV)
