@@ -157,6 +157,26 @@ __device__ __forceinline__ void add_vote(int32_t* counter, uint32_t packed, uint
 }
 #endif
 
+// ------------------------------------------------------------------ launches that overlap their predecessor's tail
+// launch_after(): the kernel's blocks may be scheduled while the previous kernel on the stream is still
+// draining (programmatic stream serialization); the kernel must call grid_dependency_wait() before it
+// touches anything, which returns once every earlier kernel has completed and its writes are visible.
+// In a kernel launched the ordinary way the wait returns at once.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ------------------------------------------------------------------ profiling
 // Optional event marks at the phase boundaries of s3gd_step (see s3gd_profile_begin).
 enum Phase : int { kPhaseStart = 0, kPhaseSampled, kPhaseFiltered, kPhaseThreshold, kPhaseEmitted, kPhaseApplied,

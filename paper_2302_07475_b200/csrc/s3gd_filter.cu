@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(1024) sample_threshold_kernel(const uint32_t* 
   extern __shared__ uint32_t s_hist[];            // kSampleBins counters
   __shared__ uint32_t s_wsum[32];
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  grid_dependency_wait();                         // (launched with launch_after: whatever ran before on the stream is done)
   if (blockIdx.x >= M) {                          // a clearing block; `zero` is 16-byte aligned, n_zero words
     const uint64_t n4 = n_zero / 4, nthr = (uint64_t)(gridDim.x - M) * 1024;
     uint4* z4 = reinterpret_cast<uint4*>(zero);
@@ -257,6 +258,7 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_kernel(const
   __shared__ uint32_t s_slow_base;
   const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, lt = lanemask_lt();
   const uint64_t n_work = (uint64_t)M * n_tiles;
+  grid_dependency_wait();                          // (launched with launch_after)
   if (blockIdx.x >= n_work) return;
   // walk (row, tile) without dividing in the loop
   uint32_t row = (uint32_t)(blockIdx.x / n_tiles), t = (uint32_t)(blockIdx.x - (uint64_t)row * n_tiles);
@@ -418,6 +420,7 @@ __global__ void __launch_bounds__(kTileThreads, kEF ? 3 : 4) filter_scan_kernel(
   __shared__ uint32_t s_direct_base;
   const uint32_t tid = threadIdx.x, lane = tid & 31;
   const uint64_t n_work = (uint64_t)M * n_tiles;
+  grid_dependency_wait();                          // (launched with launch_after)
   uint32_t pend_n = 0, pend_row = 0, pend_t = 0;   // staged survivors of the previous tile (uniform)
   uint32_t pend_base = 0;                          // thread 0: the claim made for them (may still be in flight)
   int par = 0;
@@ -610,6 +613,7 @@ __global__ void __launch_bounds__(kThreads, kBandThreadsPerSm / kThreads) filter
                                                                                 uint2* __restrict__ cand, uint32_t cap,
                                                                                 int32_t* __restrict__ counter,
                                                                                 uint32_t packed) {
+  grid_dependency_wait();                                        // (launched with launch_after)
   constexpr uint32_t kElems = (uint32_t)kThreads * 32u;          // entries per tile
   constexpr int kQueueCap = 4 * kThreads;                        // survivors of a tile the queue holds
   constexpr int kBandStage = 2 * kThreads;                       // band entries of a tile the band buffer holds
@@ -761,11 +765,9 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
     n_clear = (unsigned)sm_count() - used;
     if (n_clear < 32u) n_clear += (unsigned)sm_count();
   }
-  sample<<<(unsigned)L.M + n_clear, 1024, smem, st>>>(gbits, L.d, rows, L.n_sample, L.sample_stride, L.j_rank,
-                                                      band ? L.j_hi_rank : 0u, (uint32_t)L.K, hdr, hist, ef_err, eta,
-                                                      (uint32_t)L.M, zero_counter,
-                                                      packed ? (L.d + 3) / 4 : L.d, packed ? kPackedZero : 0u);
-  e = cudaGetLastError();
+  e = launch_after(sample, dim3((unsigned)L.M + n_clear), dim3(1024), smem, st, gbits, L.d, rows, L.n_sample,
+                   L.sample_stride, L.j_rank, band ? L.j_hi_rank : 0u, (uint32_t)L.K, hdr, hist, ef_err, eta, (uint32_t)L.M,
+                   zero_counter, packed ? (L.d + 3) / 4 : L.d, packed ? kPackedZero : 0u);
   if (e != cudaSuccess) return e;
   prof_mark(kPhaseSampled, st);
   count_launch(2);
@@ -775,15 +777,14 @@ cudaError_t launch_sample_and_filter(const uint32_t* gbits, const Layout& L, Row
     constexpr int kBandThreads = 256;
     const uint64_t tiles = (uint64_t)L.M * ((L.d + kBandThreads * 32 - 1) / (kBandThreads * 32));
     const uint64_t resident = (uint64_t)sm_count() * (kBandThreadsPerSm / kBandThreads);
-    filter_band_kernel<kBandThreads><<<(unsigned)(tiles < resident ? tiles : resident), kBandThreads, 0, st>>>(
-        gbits, L.M, L.d, rows, cand, L.cap, zero_counter, packed ? 1u : 0u);
-    return cudaGetLastError();
+    return launch_after(filter_band_kernel<kBandThreads>, dim3((unsigned)(tiles < resident ? tiles : resident)),
+                        dim3(kBandThreads), 0, st, gbits, L.M, L.d, rows, cand, L.cap, zero_counter, packed ? 1u : 0u);
   }
   const bool dense = L.dense;
   auto filter = dense ? (ef_err ? filter_scan_kernel<true> : filter_scan_kernel<false>)
                       : (ef_err ? filter_kernel<true> : filter_kernel<false>);
-  filter<<<(unsigned)blocks, kTileThreads, 0, st>>>(gbits, L.M, L.d, rows, cand, L.cap, seg, L.n_tiles, ef_err, eta);
-  return cudaGetLastError();
+  return launch_after(filter, dim3((unsigned)blocks), dim3(kTileThreads), 0, st, gbits, L.M, L.d, rows, cand, L.cap, seg,
+                      L.n_tiles, ef_err, eta);
 }
 
 }  // namespace s3gd

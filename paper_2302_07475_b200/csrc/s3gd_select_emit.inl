@@ -382,6 +382,7 @@ __global__ void __launch_bounds__(kSelThreads, 6) hist_two_pass_kernel(const uin
                                                                        uint32_t* __restrict__ hdr, int pass,
                                                                        uint2* __restrict__ bin, uint32_t bin_cap,
                                                                        EmitOut o, bool band) {
+  grid_dependency_wait();                          // (launched with launch_after)
   hist_two_pass_block(cand, cap, rows, K, hist, hdr, pass, blockIdx.x, blockIdx.y, gridDim.x, bin, bin_cap, o, band);
 }
 
@@ -533,10 +534,12 @@ cudaError_t launch_select(const float* grads, const Layout& L, void* ws, uint32_
     // bin lists only where the votes alone are wanted (the message needs positions)
     uint2* bin = reinterpret_cast<uint2*>(base + L.off_bin);
     const uint32_t bin_cap = band ? L.bin_cap : 0u;
-    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 0, bin, bin_cap, o, band);
-    S3GD_CHECK_LAUNCH();
-    hist_two_pass_kernel<<<dim3(gx_two, M), kSelThreads, 0, st>>>(cand, L.cap, rows, K, hist, hdr, 2, bin, bin_cap, o, band);
-    S3GD_CHECK_LAUNCH();
+    for (int pass = 0; pass <= 2; pass += 2) {
+      cudaError_t e = launch_after(hist_two_pass_kernel, dim3(gx_two, M), dim3(kSelThreads), 0, st, cand, L.cap, rows, K, hist,
+                                   hdr, pass, bin, bin_cap, o, band);
+      if (e != cudaSuccess) return e;
+      count_launch();
+    }
     prof_mark(kPhaseThreshold, st);
     if (bin_cap) {
       cudaError_t e = launch_select_bin(L, rows, bin, bin_cap, hdr, o, st);

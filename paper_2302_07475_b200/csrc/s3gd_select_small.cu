@@ -216,6 +216,7 @@ select_small_kernel(RowState* __restrict__ rows, const uint2* __restrict__ cand,
   __shared__ uint32_t s_sel[2];
   __shared__ uint32_t s_first[kOrdered ? kSmallThreads : 1];   // first chunk of each tile of a layout round
   const uint32_t row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, lt = lanemask_lt();
+  grid_dependency_wait();                            // (launched with launch_after)
   const RowState rs = rows[row];
   if (kBin ? rs.done != kRowBin : !row_uses_candidates(rs, o.K, cap)) return;
   if (!kBin && !fits_single_cta(rs.n_cand)) {
@@ -585,6 +586,7 @@ select_cluster_kernel(RowState* __restrict__ rows, const uint2* __restrict__ can
   __shared__ uint32_t s_sel[2];
   const uint32_t rank = cluster.block_rank();             // the launch gives the cluster C CTAs
   const uint32_t row = blockIdx.x / C, tid = threadIdx.x, lane = tid & 31;
+  grid_dependency_wait();                                 // (the launch allows an early start, as launch_after() does)
   const RowState rs = rows[row];
   const uint32_t n = rs.n_cand;
   const uint32_t per_cta = (n + C - 1) / C;
@@ -757,8 +759,7 @@ cudaError_t launch_select_small(const Layout& L, RowState* rows, const uint2* ca
   static int opted[2][kMaxDevices];
   cudaError_t e = opt_in_dynamic_smem(reinterpret_cast<const void*>(kernel), (int)kSmallSelectBytes, opted[ordered ? 1 : 0]);
   if (e != cudaSuccess) return e;
-  kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, cand, L.cap, seg, L.n_tiles, hdr, o);
-  e = cudaGetLastError();
+  e = launch_after(kernel, dim3(L.M), dim3(kSmallThreads), (size_t)need, st, rows, cand, L.cap, seg, L.n_tiles, hdr, o);
   if (e == cudaSuccess) count_launch();
   return e;
 }
@@ -771,8 +772,8 @@ cudaError_t launch_select_bin(const Layout& L, RowState* rows, const uint2* bin,
   if (e != cudaSuccess) return e;
   uint64_t need = (uint64_t)bin_cap * 8u;
   if (need > kSmallSelectBytes) need = kSmallSelectBytes;
-  kernel<<<L.M, kSmallThreads, (size_t)need, st>>>(rows, bin, bin_cap, nullptr, 0u, hdr, o);
-  e = cudaGetLastError();
+  e = launch_after(kernel, dim3(L.M), dim3(kSmallThreads), (size_t)need, st, rows, bin, bin_cap,
+                   static_cast<const uint2*>(nullptr), 0u, hdr, o);
   if (e == cudaSuccess) count_launch();
   return e;
 }
@@ -804,13 +805,15 @@ cudaError_t launch_select_cluster(const Layout& L, RowState* rows, const uint2* 
   cfg.blockDim = dim3(kSmallThreads);
   cfg.dynamicSmemBytes = (size_t)need;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;    // as launch_after()
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   e = cudaLaunchKernelEx(&cfg, kernel, rows, cand, L.cap, hdr, o);
   if (e == cudaSuccess) count_launch();
   return e;

@@ -137,6 +137,7 @@ template <bool kVec>
 __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_t* __restrict__ cw,
                                                                    float* __restrict__ x, uint64_t d, float lr,
                                                                    int8_t* __restrict__ opt_vote) {
+  grid_dependency_wait();                            // (launched with launch_after)
   const uint64_t n_words = (d + 3) / 4;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride) {
@@ -179,6 +180,7 @@ __global__ void __launch_bounds__(256) counter_apply_packed_kernel(const uint32_
 // that differs from the zero pattern.  x 16-byte aligned, no vote output.
 __global__ void __launch_bounds__(256) counter_apply_packed_sparse_kernel(const uint32_t* __restrict__ cw,
                                                                           float* __restrict__ x, uint64_t d, float lr) {
+  grid_dependency_wait();                            // (launched with launch_after)
   const uint64_t n_words = (d + 3) / 4, n_groups = n_words / 4;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   const uint64_t first = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -369,15 +371,15 @@ cudaError_t launch_counter_apply(const int32_t* counter, bool packed, float* x, 
     const uint32_t* cw = reinterpret_cast<const uint32_t*>(counter);
     if (max_votes != 0 && max_votes <= d / kSparseVotesRatio && opt_vote == nullptr && aligned(x, 16) &&
         aligned(counter, 16)) {
-      counter_apply_packed_sparse_kernel<<<grid_for((d + 15) / 16, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr);
       count_launch();
-      return cudaGetLastError();
+      return launch_after(counter_apply_packed_sparse_kernel, dim3(grid_for((d + 15) / 16, 256, sm_count() * 8)), dim3(256), 0,
+                          st, cw, x, d, lr);
     }
     const bool vecp = aligned(x, 16) && (opt_vote == nullptr || aligned(opt_vote, 4));
-    if (vecp) counter_apply_packed_kernel<true><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
-    else counter_apply_packed_kernel<false><<<grid_for((d + 3) / 4, 256, sm_count() * 8), 256, 0, st>>>(cw, x, d, lr, opt_vote);
+    const dim3 grid(grid_for((d + 3) / 4, 256, sm_count() * 8));
     count_launch();
-    return cudaGetLastError();
+    return vecp ? launch_after(counter_apply_packed_kernel<true>, grid, dim3(256), 0, st, cw, x, d, lr, opt_vote)
+                : launch_after(counter_apply_packed_kernel<false>, grid, dim3(256), 0, st, cw, x, d, lr, opt_vote);
   }
   bool vec = aligned(x, 16) && aligned(counter, 16) && (opt_vote == nullptr || aligned(opt_vote, 4)) && d >= 4;
   if (vec) {
