@@ -18,7 +18,9 @@
  *    retains a pointer.  Every buffer, including the workspace, is the caller's.
  *  - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
  *    the default stream).  No call synchronises except s3gd_device_status(),
- *    s3gd_last_device_status() and s3gd_profile_end().
+ *    s3gd_last_device_status() and s3gd_profile_end().  Stream order is kept: some kernels are
+ *    launched so that their blocks may be scheduled while the previous kernel on the stream
+ *    (the caller's included) is still draining, but they touch no memory before it has completed.
  *  - Magnitude order is the unsigned order of the fp32 bit pattern with the sign
  *    bit cleared.  Denormals are not flushed; NaN and Inf order by bit pattern.
  *  - Exactly K entries are kept per worker; equal magnitudes go to the lower
